@@ -1,0 +1,206 @@
+"""CPU oracle for the random-line-read path -- TEST INFRASTRUCTURE.
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and the CPU-baseline / reference legs of
+``bench.py`` may import this package.  It shares no code with the CUDA library and the
+product never routes through it.
+
+The arithmetic lives in ``rr_oracle.c`` (plain C, one word at a time); this module only
+compiles that file with gcc and marshals numpy arrays into it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "rr_oracle.c"
+_LIB = _HERE / "librr_oracle.so"
+
+INDEX_RANDOM = 0
+INDEX_STRIDE = 1
+SM_INACTIVE = 0xFFFF
+
+
+def build(force: bool = False) -> Path:
+    """Compile rr_oracle.c into a shared object next to it (gcc, OpenMP)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.run(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-ffp-contract=off",
+             str(_SRC), "-o", str(tmp), "-lm"],
+            check=True,
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(str(build()))
+        u64, u32, i32 = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int32
+        p = ctypes.c_void_p
+        lib.orc_sm64.restype = u64
+        lib.orc_sm64.argtypes = [u64]
+        lib.orc_word.restype = u32
+        lib.orc_word.argtypes = [u64]
+        lib.orc_fill.restype = None
+        lib.orc_fill.argtypes = [p, u64, u64]
+        lib.orc_warp_key.restype = u64
+        lib.orc_warp_key.argtypes = [u64, u64]
+        lib.orc_draw.restype = u64
+        lib.orc_draw.argtypes = [u64, u64, u64]
+        lib.orc_line.restype = u64
+        lib.orc_line.argtypes = [u32, u64, u64, u64, u64, u64, u64]
+        lib.orc_warp_checksum.restype = None
+        lib.orc_warp_checksum.argtypes = [u32, u64, u64, u64, u64, u64, u32, u64, u64, p, p]
+        lib.orc_read_logical.restype = i32
+        lib.orc_read_logical.argtypes = [u64, u32, u32, u64, u64, u64, u64, p]
+        lib.orc_read_per_sm.restype = i32
+        lib.orc_read_per_sm.argtypes = [u64, u32, u32, u32, u32, u64, u64, u64, p, p, p, u32, p]
+        lib.orc_make_windows.restype = i32
+        lib.orc_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p, p]
+        lib.orc_cluster.restype = i32
+        lib.orc_cluster.argtypes = [p, u32, p, p, p, p]
+        lib.orc_reach.restype = i32
+        lib.orc_reach.argtypes = [p, p, u32, p, p]
+        _lib = lib
+    return _lib
+
+
+class OracleError(ValueError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle rejected its arguments (code {code})")
+        self.code = code
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def sm64(x: int) -> int:
+    return int(_load().orc_sm64(x & 0xFFFFFFFFFFFFFFFF))
+
+
+def word(i: int) -> int:
+    return int(_load().orc_word(i))
+
+
+def fill(first_word: int, n_words: int) -> np.ndarray:
+    out = np.empty(n_words, dtype=np.uint32)
+    _load().orc_fill(_ptr(out), first_word, n_words)
+    return out
+
+
+def warp_key(seed: int, v: int) -> int:
+    return int(_load().orc_warp_key(seed, v))
+
+
+def draw(seed: int, v: int, i: int) -> int:
+    return int(_load().orc_draw(seed, v, i))
+
+
+def line(seed: int, v: int, i: int, base: int, n: int, index_mode: int = INDEX_RANDOM,
+         n_warps_total: int = 1) -> int:
+    return int(_load().orc_line(index_mode, seed, v, n_warps_total, i, base, n))
+
+
+def warp_checksum(seed: int, v: int, first_read: int, reads: int, W: int, base: int, n: int,
+                  index_mode: int = INDEX_RANDOM, n_warps_total: int = 1):
+    x = ctypes.c_uint32()
+    s = ctypes.c_uint32()
+    _load().orc_warp_checksum(index_mode, seed, v, n_warps_total, first_read, reads, W, base, n,
+                              ctypes.byref(x), ctypes.byref(s))
+    return int(x.value), int(s.value)
+
+
+def read_logical(region_bytes: int, W: int, n_warps: int, reads: int, seed: int,
+                 first_read: int = 0, index_mode: int = INDEX_RANDOM) -> np.ndarray:
+    """Checksums {X, S} of logical warps 0..n_warps-1 over the whole region: (n_warps, 2) uint32."""
+    out = np.zeros((n_warps, 2), dtype=np.uint32)
+    rc = _load().orc_read_logical(region_bytes, W, index_mode, n_warps, first_read, reads, seed,
+                                  _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def read_per_sm(region_bytes: int, W: int, nsm: int, wps: int, reads: int, seed: int,
+                group_of_sm=None, windows=None, first_read: int = 0,
+                index_mode: int = INDEX_RANDOM) -> np.ndarray:
+    """Checksums of warps v = smid*wps + warp: (nsm*wps, 2) uint32.
+
+    ``windows`` is an (n_groups, 2) array of {base_line, n_lines}."""
+    out = np.zeros((nsm * wps, 2), dtype=np.uint32)
+    g = wb = wn = None
+    ng = 0
+    if group_of_sm is not None:
+        g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+        if g.shape != (nsm,):
+            raise OracleError(-1)
+        w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+        wb = np.ascontiguousarray(w[:, 0])
+        wn = np.ascontiguousarray(w[:, 1])
+        ng = w.shape[0]
+    rc = _load().orc_read_per_sm(region_bytes, W, index_mode, nsm, wps, first_read, reads, seed,
+                                 _ptr(g), _ptr(wb), _ptr(wn), ng, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int, policy: int = 0,
+                 seed: int = 0):
+    """Windows per group as (n_groups, 2) uint32 {base_line, n_lines}, and the coverage fraction."""
+    wb = np.zeros(n_groups, dtype=np.uint32)
+    wn = np.zeros(n_groups, dtype=np.uint32)
+    cov = ctypes.c_double()
+    rc = _load().orc_make_windows(region_bytes, W, window_bytes, n_groups, policy, seed, _ptr(wb),
+                                  _ptr(wn), ctypes.byref(cov))
+    if rc != 0:
+        raise OracleError(rc)
+    return np.stack([wb, wn], axis=1), float(cov.value)
+
+
+def cluster(T):
+    """SM x SM throughput matrix -> (group_of_sm int32[n], n_groups, confidence, heights[n-1])."""
+    T = np.ascontiguousarray(T, dtype=np.float32)
+    n = T.shape[0]
+    if T.shape != (n, n):
+        raise OracleError(-1)
+    groups = np.zeros(n, dtype=np.int32)
+    heights = np.zeros(max(n - 1, 1), dtype=np.float64)
+    ng = ctypes.c_uint32()
+    conf = ctypes.c_double()
+    rc = _load().orc_cluster(_ptr(T), n, _ptr(groups), ctypes.byref(ng), ctypes.byref(conf),
+                             _ptr(heights))
+    if rc != 0:
+        raise OracleError(rc)
+    return groups, int(ng.value), float(conf.value), heights[: n - 1]
+
+
+def reach(size_bytes, gbps):
+    """(cliff_exists, plateau GB/s, reach bytes) from an increasing size sweep."""
+    s = np.ascontiguousarray(size_bytes, dtype=np.uint64)
+    g = np.ascontiguousarray(gbps, dtype=np.float64)
+    plateau = ctypes.c_double()
+    r = ctypes.c_uint64()
+    rc = _load().orc_reach(_ptr(s), _ptr(g), len(s), ctypes.byref(plateau), ctypes.byref(r))
+    if rc < 0:
+        raise OracleError(rc)
+    return bool(rc), float(plateau.value), int(r.value)
+
+
+def n_threads() -> int:
+    """Threads the OpenMP loops will use (host cores available to this process)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env.split(",")[0])
+    return len(os.sched_getaffinity(0))

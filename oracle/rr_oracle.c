@@ -1,0 +1,436 @@
+/*
+ * rr_oracle.c -- plain CPU definition of the random-line-read path.
+ *
+ * TEST INFRASTRUCTURE.  Only the tests, the smoke check and the CPU-baseline leg
+ * of the benchmark may call this file.  It shares no source, header, table or
+ * constant generator with the CUDA library; the product never falls back to it.
+ *
+ * What it defines (the paper gives prose only, so every definition below is a
+ * stated reading of that prose):
+ *   - Section 2.1 "Basic benchmark": every warp reads random coalesced arrays of
+ *     32 words (32-, 64- or 128-bit) inside a memory region; here the region has
+ *     known contents (a hash of the word index), the random line comes from a
+ *     counter-based generator, and what is read is folded into two checksums per
+ *     warp so that a reader can prove which lines were touched.
+ *   - Section 2.1, second experiment and Section 2.4: all warps of an SM (of an SM
+ *     group) are held to one chunk (window) of the region.
+ *   - Section 2.2: the SM x SM pair-throughput matrix is rearranged into groups;
+ *     here: average-linkage agglomeration with a largest-gap cut.
+ *
+ * Everything is written as the definition, one word at a time, with no blocking,
+ * fusion or reordering.  The only parallelism is an OpenMP loop over warps, which
+ * are independent by definition.
+ *
+ * Pins (see tests/test_oracle_*.py): the public SplitMix64 output streams, a
+ * big-integer brute force over tiny materialised buffers, window invariants,
+ * the width identity, a sequential mode that must fold the whole buffer, draw
+ * statistics, and planted partitions for the clustering.
+ * Parity unpinned: orc_reach() thresholds (0.8 / 0.9 of the plateau) are a
+ * reading with no external truth; only their bookkeeping is tested.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_ERR_ARG (-1)
+#define ORC_ERR_RANGE (-3)
+#define ORC_ERR_MAP (-4)
+
+#define ORC_INDEX_RANDOM 0u
+#define ORC_INDEX_STRIDE 1u
+#define ORC_SM_INACTIVE 0xFFFFu
+
+/* ---- O1: mixing function and buffer contents --------------------------------
+ * sm64(x) is the first output of a SplitMix64 generator whose state is x:
+ * add the golden-ratio increment, then the three-step finaliser.              */
+static const uint64_t ORC_GAMMA = 0x9E3779B97F4A7C15ULL;
+
+uint64_t orc_sm64(uint64_t x)
+{
+    uint64_t z = x + ORC_GAMMA;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+/* Contents of 32-bit word i of the buffer (i counts from the buffer start). */
+uint32_t orc_word(uint64_t i)
+{
+    return (uint32_t)(orc_sm64(i) & 0xFFFFFFFFULL);
+}
+
+void orc_fill(uint32_t *dst, uint64_t first_word, uint64_t n_words)
+{
+    for (uint64_t k = 0; k < n_words; ++k)
+        dst[k] = orc_word(first_word + k);
+}
+
+/* ---- O2: line index ----------------------------------------------------------
+ * A keyed, random-access SplitMix64 stream per logical warp v:
+ *   k_seed = sm64(seed);  k_v = sm64(k_seed ^ v);  r(seed,v,i) = sm64(k_v + i*gamma)
+ * i.e. the i-th output (0-based) of a SplitMix64 generator with state k_v.      */
+uint64_t orc_warp_key(uint64_t seed, uint64_t v)
+{
+    return orc_sm64(orc_sm64(seed) ^ v);
+}
+
+uint64_t orc_draw(uint64_t seed, uint64_t v, uint64_t i)
+{
+    return orc_sm64(orc_warp_key(seed, v) + i * ORC_GAMMA);
+}
+
+/* Line (in units of 128*W bytes from the buffer start) read i of warp v hits.
+ * RANDOM: base + (r mod n).  STRIDE (sequential control, Section 2.1 last
+ * paragraph): base + ((i * n_warps_total + v) mod n).                          */
+uint64_t orc_line(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t n_warps_total,
+                  uint64_t i, uint64_t base, uint64_t n)
+{
+    uint64_t idx;
+    if (index_mode == ORC_INDEX_STRIDE)
+        idx = (i * n_warps_total + v) % n;
+    else
+        idx = orc_draw(seed, v, i) % n;
+    return base + idx;
+}
+
+/* ---- O3: what one warp reads and folds ---------------------------------------
+ * Lane l of the warp reads W consecutive 32-bit words starting at word
+ * line*32W + l*W; every 32-bit word is folded separately:
+ *   X = xor of all words, S = sum of all words mod 2^32,
+ * over 32 lanes, W words, R reads (a line drawn twice counts twice).            */
+void orc_warp_checksum(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t n_warps_total,
+                       uint64_t first_read, uint64_t reads, uint32_t W,
+                       uint64_t base, uint64_t n, uint32_t *X, uint32_t *S)
+{
+    uint32_t x = 0, s = 0;
+    for (uint64_t t = 0; t < reads; ++t) {
+        uint64_t line = orc_line(index_mode, seed, v, n_warps_total, first_read + t, base, n);
+        for (uint32_t lane = 0; lane < 32; ++lane) {
+            for (uint32_t w = 0; w < W; ++w) {
+                uint64_t j = line * 32u * W + (uint64_t)lane * W + w;
+                uint32_t word = orc_word(j);
+                x ^= word;
+                s += word;
+            }
+        }
+    }
+    *X = x;
+    *S = s;
+}
+
+static int orc_width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
+
+/* Logical-warp mode: v = 0 .. n_warps-1, window = the whole region.
+ * out holds n_warps pairs {X, S}.                                               */
+int32_t orc_read_logical(uint64_t region_bytes, uint32_t W, uint32_t index_mode,
+                         uint64_t n_warps, uint64_t first_read, uint64_t reads,
+                         uint64_t seed, uint32_t *out)
+{
+    if (!orc_width_ok(W) || index_mode > 1 || !out) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    int64_t nw = (int64_t)n_warps;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v)
+        orc_warp_checksum(index_mode, seed, (uint64_t)v, n_warps, first_read, reads, W, 0, L,
+                          &out[2 * v], &out[2 * v + 1]);
+    return ORC_OK;
+}
+
+/* Per-SM mode: v = smid*wps + warp; window = windows[group_of_sm[smid]] (whole
+ * region when group_of_sm is NULL); inactive SMs (0xFFFF) give {0,0}.
+ * out holds nsm*wps pairs.                                                      */
+int32_t orc_read_per_sm(uint64_t region_bytes, uint32_t W, uint32_t index_mode,
+                        uint32_t nsm, uint32_t wps, uint64_t first_read, uint64_t reads,
+                        uint64_t seed, const uint16_t *group_of_sm,
+                        const uint32_t *win_base, const uint32_t *win_n, uint32_t n_groups,
+                        uint32_t *out)
+{
+    if (!orc_width_ok(W) || index_mode > 1 || !out || nsm == 0 || wps == 0) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    if (group_of_sm) {
+        if (!win_base || !win_n || n_groups == 0) return ORC_ERR_ARG;
+        for (uint32_t g = 0; g < n_groups; ++g)
+            if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
+        for (uint32_t s = 0; s < nsm; ++s)
+            if (group_of_sm[s] != ORC_SM_INACTIVE && group_of_sm[s] >= n_groups) return ORC_ERR_MAP;
+    }
+    uint64_t total = (uint64_t)nsm * wps;
+    int64_t nw = (int64_t)total;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t sm = (uint32_t)(v / wps);
+        uint64_t base = 0, n = L;
+        if (group_of_sm) {
+            if (group_of_sm[sm] == ORC_SM_INACTIVE) {
+                out[2 * v] = 0;
+                out[2 * v + 1] = 0;
+                continue;
+            }
+            base = win_base[group_of_sm[sm]];
+            n = win_n[group_of_sm[sm]];
+        }
+        orc_warp_checksum(index_mode, seed, (uint64_t)v, total, first_read, reads, W, base, n,
+                          &out[2 * v], &out[2 * v + 1]);
+    }
+    return ORC_OK;
+}
+
+/* ---- O4: windows (Section 1.3 "half the memory for simplicity", Section 2.4) ---
+ * L lines are cut into K = ceil(L / S_lines) chunks of floor(L/K) lines, the last
+ * one running to L.  policy 0: group g takes chunk g mod K.  policy 1 (the
+ * paper's naive control, one "group" per SM): chunk sm64(seed ^ g) mod K.
+ * coverage = distinct chunks used / K.                                          */
+int32_t orc_make_windows(uint64_t region_bytes, uint32_t W, uint64_t window_bytes,
+                         uint32_t n_groups, uint32_t policy, uint64_t seed,
+                         uint32_t *win_base, uint32_t *win_n, double *coverage)
+{
+    if (!orc_width_ok(W) || n_groups == 0 || policy > 1 || !win_base || !win_n) return ORC_ERR_ARG;
+    uint64_t line_bytes = 128ull * W;
+    uint64_t L = region_bytes / line_bytes;
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    uint64_t S = window_bytes / line_bytes;
+    if (S < 1) S = 1;
+    if (S > L) S = L;
+    uint64_t K = (L + S - 1) / S;
+    uint64_t chunk = L / K;
+    unsigned char *used = (unsigned char *)calloc((size_t)K, 1);
+    if (!used) return ORC_ERR_ARG;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        uint64_t c = (policy == 1) ? (orc_sm64(seed ^ (uint64_t)g) % K) : ((uint64_t)g % K);
+        uint64_t lo = c * chunk;
+        uint64_t hi = (c == K - 1) ? L : (c + 1) * chunk;
+        win_base[g] = (uint32_t)lo;
+        win_n[g] = (uint32_t)(hi - lo);
+        used[c] = 1;
+    }
+    uint64_t distinct = 0;
+    for (uint64_t c = 0; c < K; ++c) distinct += used[c];
+    free(used);
+    if (coverage) *coverage = (double)distinct / (double)K;
+    return ORC_OK;
+}
+
+/* ---- O5: SM x SM matrix -> groups (Section 2.2, Figures 2 and 3) ---------------
+ * 1. symmetrise off-diagonal entries in double: t = (T_ij + T_ji) / 2
+ * 2. quantise: q = rint(t * 2^20 / lower-median(t)), clamped to 2^32-1
+ * 3. average linkage on q (small q = contended = close): exact integer pair sums,
+ *    means compared by cross-multiplication, ties -> smallest (a,b); a cluster is
+ *    named by its smallest member; height of a merge = sum / (na*nb) in double
+ * 4. cut: apply the first k merges, k chosen among cuts leaving 2..floor(n/3)
+ *    clusters to maximise h[k] - h[k-1]; the first maximum wins
+ * 5. null rule: sigma = 1.4826 * MAD of the q of pairs in different clusters after
+ *    the cut, divided by sqrt of the number of pairs averaged in merge k (so it
+ *    is the noise of the height that defines the gap); gap < 4 sigma -> one group
+ * 6. labels: groups numbered by their smallest SM id
+ * heights (optional) receives the n-1 merge heights.                            */
+static int cmp_double(const void *a, const void *b)
+{
+    double x = *(const double *)a, y = *(const double *)b;
+    return (x > y) - (x < y);
+}
+static int cmp_u32(const void *a, const void *b)
+{
+    uint32_t x = *(const uint32_t *)a, y = *(const uint32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int32_t orc_cluster(const float *T, uint32_t n, int32_t *group_of_sm, uint32_t *n_groups,
+                    double *confidence, double *heights)
+{
+    if (!T || !group_of_sm || !n_groups || n < 2 || n > 256) return ORC_ERR_ARG;
+    size_t m = (size_t)n * (n - 1) / 2;
+    double *t = (double *)malloc(sizeof(double) * (size_t)n * n);
+    double *sorted = (double *)malloc(sizeof(double) * m);
+    uint32_t *q = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)n * n);
+    uint64_t *sum = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)n * n);
+    uint32_t *size = (uint32_t *)malloc(sizeof(uint32_t) * n);
+    uint32_t *alive = (uint32_t *)malloc(sizeof(uint32_t) * n);
+    uint32_t *merge_a = (uint32_t *)malloc(sizeof(uint32_t) * n);
+    uint32_t *merge_b = (uint32_t *)malloc(sizeof(uint32_t) * n);
+    uint64_t *merge_pairs = (uint64_t *)malloc(sizeof(uint64_t) * n);
+    double *h = (double *)malloc(sizeof(double) * n);
+    uint32_t *between = (uint32_t *)malloc(sizeof(uint32_t) * (m ? m : 1));
+    int32_t rc = ORC_OK;
+    if (!t || !sorted || !q || !sum || !size || !alive || !merge_a || !merge_b || !merge_pairs ||
+        !h || !between) {
+        rc = ORC_ERR_ARG;
+        goto done;
+    }
+
+    /* 1. symmetrise, validate */
+    {
+        size_t k = 0;
+        for (uint32_t i = 0; i < n; ++i)
+            for (uint32_t j = i + 1; j < n; ++j) {
+                double a = (double)T[(size_t)i * n + j], b = (double)T[(size_t)j * n + i];
+                if (!(a > 0.0) || !(b > 0.0) || isinf(a) || isinf(b)) {
+                    rc = ORC_ERR_ARG;
+                    goto done;
+                }
+                double s = (a + b) * 0.5;
+                t[(size_t)i * n + j] = s;
+                t[(size_t)j * n + i] = s;
+                sorted[k++] = s;
+            }
+    }
+    /* 2. quantise against the lower median */
+    qsort(sorted, m, sizeof(double), cmp_double);
+    {
+        double med = sorted[(m - 1) / 2];
+        for (uint32_t i = 0; i < n; ++i)
+            for (uint32_t j = 0; j < n; ++j) {
+                if (i == j) {
+                    q[(size_t)i * n + j] = 0;
+                    continue;
+                }
+                double r = rint(t[(size_t)i * n + j] * 1048576.0 / med);
+                q[(size_t)i * n + j] = (r >= 4294967295.0) ? 0xFFFFFFFFu : (uint32_t)r;
+            }
+    }
+    /* 3. average linkage */
+    for (uint32_t i = 0; i < n; ++i) {
+        size[i] = 1;
+        alive[i] = 1;
+        for (uint32_t j = 0; j < n; ++j) sum[(size_t)i * n + j] = q[(size_t)i * n + j];
+    }
+    for (uint32_t step = 0; step + 1 < n; ++step) {
+        int have = 0;
+        uint32_t ba = 0, bb = 0;
+        uint64_t bs = 0, bp = 1;
+        for (uint32_t a = 0; a < n; ++a) {
+            if (!alive[a]) continue;
+            for (uint32_t b = a + 1; b < n; ++b) {
+                if (!alive[b]) continue;
+                uint64_t s = sum[(size_t)a * n + b];
+                uint64_t p = (uint64_t)size[a] * size[b];
+                /* s/p < bs/bp  <=>  s*bp < bs*p  (all < 2^60 for n <= 256) */
+                if (!have || s * bp < bs * p) {
+                    have = 1;
+                    ba = a;
+                    bb = b;
+                    bs = s;
+                    bp = p;
+                }
+            }
+        }
+        merge_a[step] = ba;
+        merge_b[step] = bb;
+        merge_pairs[step] = bp;
+        h[step] = (double)bs / (double)bp;
+        for (uint32_t c = 0; c < n; ++c) {
+            if (!alive[c] || c == ba || c == bb) continue;
+            uint64_t s = sum[(size_t)ba * n + c] + sum[(size_t)bb * n + c];
+            sum[(size_t)ba * n + c] = s;
+            sum[(size_t)c * n + ba] = s;
+        }
+        size[ba] += size[bb];
+        alive[bb] = 0;
+    }
+    if (heights)
+        for (uint32_t k = 0; k + 1 < n; ++k) heights[k] = h[k];
+
+    /* 4. cut */
+    for (uint32_t i = 0; i < n; ++i) group_of_sm[i] = 0;
+    *n_groups = 1;
+    if (confidence) *confidence = 0.0;
+    {
+        uint32_t max_clusters = n / 3;
+        if (max_clusters < 2) goto done; /* too few SMs for a group level */
+        uint32_t k_lo = n - max_clusters, k_hi = n - 2, best_k = 0;
+        double best_gap = -1.0;
+        for (uint32_t k = k_lo; k <= k_hi; ++k) {
+            double gap = h[k] - h[k - 1];
+            if (gap > best_gap) {
+                best_gap = gap;
+                best_k = k;
+            }
+        }
+        /* replay the first best_k merges; parent[] by smallest member */
+        uint32_t *rep = alive; /* reuse: representative of each SM */
+        for (uint32_t i = 0; i < n; ++i) rep[i] = i;
+        for (uint32_t k = 0; k < best_k; ++k)
+            for (uint32_t i = 0; i < n; ++i)
+                if (rep[i] == merge_b[k]) rep[i] = merge_a[k];
+        /* 5. null rule */
+        size_t nb = 0;
+        for (uint32_t i = 0; i < n; ++i)
+            for (uint32_t j = i + 1; j < n; ++j)
+                if (rep[i] != rep[j]) between[nb++] = q[(size_t)i * n + j];
+        qsort(between, nb, sizeof(uint32_t), cmp_u32);
+        uint32_t bmed = between[(nb - 1) / 2];
+        for (size_t k = 0; k < nb; ++k)
+            between[k] = between[k] > bmed ? between[k] - bmed : bmed - between[k];
+        qsort(between, nb, sizeof(uint32_t), cmp_u32);
+        double mad = (double)between[(nb - 1) / 2];
+        double sigma = (1.4826 * mad) / sqrt((double)merge_pairs[best_k]);
+        double conf = sigma > 0.0 ? best_gap / sigma : (best_gap > 0.0 ? INFINITY : 0.0);
+        if (confidence) *confidence = conf;
+        if (!(best_gap >= 4.0 * sigma) || !(best_gap > 0.0)) goto done; /* one group */
+        /* 6. canonical labels: representatives are smallest members */
+        uint32_t G = 0;
+        for (uint32_t i = 0; i < n; ++i)
+            if (rep[i] == i) merge_pairs[i] = G++; /* reuse as label-of-representative */
+        for (uint32_t i = 0; i < n; ++i) group_of_sm[i] = (int32_t)merge_pairs[rep[i]];
+        *n_groups = G;
+    }
+done:
+    free(t);
+    free(sorted);
+    free(q);
+    free(sum);
+    free(size);
+    free(alive);
+    free(merge_a);
+    free(merge_b);
+    free(merge_pairs);
+    free(h);
+    free(between);
+    return rc;
+}
+
+/* ---- O6: plateau, cliff, reach from a (size, GB/s) sweep (Section 2.1, Fig. 1) ---
+ * plateau = median GB/s over 4 GiB <= N <= 32 GiB (upper of the two middle values
+ * is NOT averaged: lower median); a cliff exists iff some larger N has GB/s below
+ * 0.8 plateau; reach = largest N with GB/s >= 0.9 plateau below the first such N.
+ * Returns 1 and *reach_bytes if a cliff exists, 0 if absent.                     */
+int32_t orc_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
+                  double *plateau, uint64_t *reach_bytes)
+{
+    if (!size_bytes || !gbps || n_points == 0 || !plateau || !reach_bytes) return ORC_ERR_ARG;
+    double *mid = (double *)malloc(sizeof(double) * n_points);
+    if (!mid) return ORC_ERR_ARG;
+    uint32_t nm = 0;
+    const uint64_t GiB = 1ull << 30;
+    for (uint32_t k = 0; k < n_points; ++k) {
+        if (k && size_bytes[k] <= size_bytes[k - 1]) {
+            free(mid);
+            return ORC_ERR_ARG; /* sizes must increase */
+        }
+        if (size_bytes[k] >= 4 * GiB && size_bytes[k] <= 32 * GiB) mid[nm++] = gbps[k];
+    }
+    if (nm == 0) {
+        free(mid);
+        return ORC_ERR_RANGE;
+    }
+    qsort(mid, nm, sizeof(double), cmp_double);
+    double P = mid[(nm - 1) / 2];
+    free(mid);
+    *plateau = P;
+    *reach_bytes = 0;
+    int32_t cliff = 0;
+    uint32_t first_bad = n_points;
+    for (uint32_t k = 0; k < n_points; ++k)
+        if (size_bytes[k] > 32 * GiB && gbps[k] < 0.8 * P) {
+            cliff = 1;
+            first_bad = k;
+            break;
+        }
+    for (uint32_t k = 0; k < first_bad; ++k)
+        if (gbps[k] >= 0.9 * P) *reach_bytes = size_bytes[k];
+    return cliff;
+}

@@ -1,0 +1,90 @@
+"""Pins the oracle's hash, key stream, line indices and checksums to values it did not produce:
+the public SplitMix64 streams and an independent big-integer derivation (tests/golden)."""
+import numpy as np
+import pytest
+
+import oracle
+
+GAMMA = 0x9E3779B97F4A7C15
+M64 = (1 << 64) - 1
+
+
+def _parse_int(tok):
+    return int(tok, 16) if tok.lower().startswith("0x") else int(tok)
+
+
+def test_public_splitmix64_streams(golden_dir):
+    n_checked = 0
+    for raw in (golden_dir / "splitmix64_public.txt").read_text().splitlines():
+        if not raw.strip() or raw.startswith("#"):
+            continue
+        seed_s, outs = raw.split(":")
+        state = _parse_int(seed_s.strip())
+        for tok in outs.split():
+            # sm64(x) = first output of a generator whose state is x; the next state is x + gamma
+            assert oracle.sm64(state) == _parse_int(tok)
+            state = (state + GAMMA) & M64
+            n_checked += 1
+    assert n_checked == 8
+
+
+def test_counter_form_reproduces_public_stream(golden_dir):
+    # r(seed, v, i) = sm64(k_v + i*gamma): with the key forced to 0 this must be the public
+    # seed-0 stream, which pins the "+ i*gamma" counter form (not i, not i*anything else).
+    line = [l for l in (golden_dir / "splitmix64_public.txt").read_text().splitlines()
+            if l.startswith("0 :")][0]
+    expect = [_parse_int(t) for t in line.split(":")[1].split()]
+    got = [oracle.sm64((0 + i * GAMMA) & M64) for i in range(len(expect))]
+    assert got == expect
+
+
+def _records(golden_dir):
+    for raw in (golden_dir / "derived_kats.txt").read_text().splitlines():
+        if not raw.strip() or raw.startswith("#"):
+            continue
+        head, vals = raw.split(":")
+        yield head.split(), vals.split()
+
+
+def test_derived_known_answers(golden_dir):
+    kinds = set()
+    for head, vals in _records(golden_dir):
+        kind = head[0]
+        kinds.add(kind)
+        if kind == "word":
+            i0 = int(head[1])
+            for k, tok in enumerate(vals):
+                assert oracle.word(i0 + k) == int(tok, 16)
+        elif kind == "sm64":
+            assert oracle.sm64(int(head[1], 16)) == int(vals[0], 16)
+        elif kind == "fold":
+            a, b = int(head[1]), int(head[2])
+            w = oracle.fill(a, b - a + 1)
+            assert int(np.bitwise_xor.reduce(w)) == int(vals[0], 16)
+            assert int(w.astype(np.uint64).sum() & 0xFFFFFFFF) == int(vals[1], 16)
+        elif kind == "key":
+            assert oracle.warp_key(int(head[1]), int(head[2])) == int(vals[0], 16)
+        elif kind == "draw":
+            seed, v, i0 = map(int, head[1:4])
+            for k, tok in enumerate(vals):
+                assert oracle.draw(seed, v, i0 + k) == int(tok, 16)
+        elif kind == "lines":
+            seed, v, base, n = map(int, head[1:5])
+            for k, tok in enumerate(vals):
+                assert oracle.line(seed, v, k, base, n) == int(tok)
+        elif kind == "sum":
+            seed, v, W, reads, base, n = map(int, head[1:7])
+            assert oracle.warp_checksum(seed, v, 0, reads, W, base, n) == (
+                int(vals[0], 16), int(vals[1], 16))
+        else:
+            pytest.fail(f"unknown record {kind}")
+    assert kinds == {"word", "sm64", "fold", "key", "draw", "lines", "sum"}
+
+
+def test_cfg0_batch_matches_kats(golden_dir):
+    # the batch entry point (what the GPU is compared with) against the per-warp KATs
+    out = oracle.read_logical(1 << 30, 1, 1 << 16, 16, seed=1)
+    assert tuple(out[0]) == (0x2A95F6CF, 0x0ECE9EAF)
+    assert tuple(out[1]) == (0x64D363B4, 0x790CA7EE)
+    assert tuple(out[2]) == (0x5AF2F0EC, 0x11B53B6C)
+    assert tuple(out[65535]) == (0xA8E997CD, 0xE4F3550B)
