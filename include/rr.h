@@ -1,0 +1,230 @@
+/*
+ * rr.h -- C ABI of librr: warp-coalesced random cache-line reads over the whole HBM with
+ * SM resource groups held to address windows (arXiv 2405.11425, written for B200 / sm_100a).
+ *
+ * Conventions that hold for every entry point
+ *   - extern "C"; plain pointers and sizes.  Each pointer is marked DEVICE or HOST below.
+ *   - Every function returns an int32_t status: RR_OK (0) or a negative RR_ERR_* code.  Nothing
+ *     throws, aborts or exits.  rr_strerror() names a code; rr_last_cuda_error() gives the text
+ *     of the last CUDA failure seen by the calling thread (for RR_ERR_CUDA).
+ *   - The caller owns all device memory (region buffer, outputs, scratch).  Unless an entry
+ *     point says otherwise the library allocates nothing on the device and keeps no state
+ *     between calls.  Host arrays are borrowed for the duration of the call only.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Arguments are validated on the host before any CUDA call: a call that returns RR_ERR_ARG,
+ *     RR_ERR_ALIGN, RR_ERR_RANGE or RR_ERR_MAP has launched nothing.
+ *   - Units: a "word" is 32 bits; a "line" is 128*W bytes (W = words per lane = 1, 2 or 4),
+ *     aligned to its own size, counted from the start of the buffer; GB/s = 1e9 bytes/s.
+ *
+ * Definitions shared by several entry points (the paper gives prose only; these are the
+ * readings this library implements)
+ *   sm64(x)      = first output of a SplitMix64 generator whose state is x (add
+ *                  0x9E3779B97F4A7C15, then the 30/27/31 xor-shift-multiply finaliser)
+ *   word(i)      = low 32 bits of sm64(i)                  -- contents of buffer word i
+ *   k_v          = sm64(sm64(seed) ^ v)                    -- key of logical warp v
+ *   r(seed,v,i)  = sm64(k_v + i * 0x9E3779B97F4A7C15)      -- i-th draw of warp v
+ *   line(v,i)    = base + (r mod n)   for a window of n lines starting at line `base`
+ *                  (RR_INDEX_STRIDE: base + ((i * V + v) mod n), V = warps in the call)
+ *   checksum     = {X, S}: X = xor, S = sum mod 2^32 of every 32-bit word the warp read
+ */
+#ifndef RR_H_
+#define RR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ---- */
+#define RR_OK 0
+#define RR_ERR_ARG (-1)          /* NULL / out-of-domain argument                               */
+#define RR_ERR_ALIGN (-2)        /* buffer not 512-byte aligned, output not 8-byte aligned      */
+#define RR_ERR_RANGE (-3)        /* region shorter than a line, >= 2^32 lines, window past end  */
+#define RR_ERR_MAP (-4)          /* SM->group map names a group >= n_groups, or no SM is active */
+#define RR_ERR_CUDA (-5)         /* a CUDA call failed; see rr_last_cuda_error()                */
+#define RR_ERR_SM_UNCOVERED (-6) /* an active SM never received a block                         */
+#define RR_ERR_TIMEOUT (-7)      /* reserved: a bounded device-side wait ran out                */
+#define RR_ERR_CHECK (-8)        /* checked variant saw an address outside its window; the      */
+                                 /* offending loads were skipped                                */
+#define RR_ERR_UNSUPPORTED (-9)  /* device is not the one this library was built for            */
+
+/* ---- limits ---- */
+#define RR_MAX_SM 256u      /* SM ids the tables can hold (B200 has 148)                       */
+#define RR_MAX_GROUPS 256u  /* one window per group; the naive control uses one group per SM   */
+#define RR_MAX_WARPS_PER_SM 64u
+#define RR_SM_INACTIVE 0xFFFFu
+
+/* ---- enums (plain integers in the structs) ---- */
+#define RR_MODE_LOGICAL 0u /* v = global warp index 0..n_warps-1, window = whole region        */
+#define RR_MODE_PER_SM 1u  /* v = smid * warps_per_sm + warp, window by SM group               */
+#define RR_INDEX_RANDOM 0u
+#define RR_INDEX_STRIDE 1u
+#define RR_VARIANT_LDG 0u         /* ld.global.nc.L1::no_allocate vector loads                  */
+#define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
+
+const char *rr_strerror(int32_t code);
+const char *rr_last_cuda_error(void);
+
+/* ---- device facts ------------------------------------------------------------------------
+ * Paper, Section 1.1: the %smid / %nsmid registers are the only layout facts a program gets.
+ * Fills *out (HOST) for the current device.  nsm_reg is %nsmid read by a one-thread kernel.
+ * theoretical_gbps = 2 * memory clock * bus width / 8.                                        */
+typedef struct {
+    uint32_t nsm_prop;       /* cudaDeviceProp::multiProcessorCount                            */
+    uint32_t nsm_reg;        /* %nsmid                                                         */
+    uint32_t cc_major, cc_minor;
+    uint64_t free_bytes, total_bytes;
+    uint32_t mem_clock_khz, bus_width_bits;
+    uint64_t l2_bytes;
+    uint32_t smem_per_sm, smem_per_block_optin;
+    double theoretical_gbps;
+    char name[64];
+    char uuid[40];           /* 32 hex digits, NUL-terminated                                  */
+} rr_device_info_t;
+int32_t rr_device_info(rr_device_info_t *out /*HOST*/);
+
+/* ---- scratch ------------------------------------------------------------------------------
+ * Bytes of DEVICE scratch rr_random_read / rr_probe_pair / rr_cluster need (claim table,
+ * status words, per-block timing records, clustering work arrays).  16-byte aligned.  The
+ * library clears what must start at zero; the contents after a call are what
+ * rr_read_report() decodes.  One scratch buffer must not be shared by calls that overlap.    */
+size_t rr_scratch_bytes(void);
+
+/* ---- A1: fill -----------------------------------------------------------------------------
+ * buf[i] = word(i) for i in [0, n_words).  buf: DEVICE, 512-byte aligned, n_words*4 bytes.
+ * Asynchronous on `stream`.  n_words = 0 is a no-op.                                          */
+int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
+
+/* ---- A2-A5, A9: random line reads ---------------------------------------------------------
+ * Paper, Section 2.1 ("every warp reads random coalesced arrays of 32 32-bit words in a memory
+ * region of varying size"; 64- and 128-bit words), Section 2.1 second experiment and Section
+ * 2.4 (all warps of an SM / of an SM group read inside one chunk).
+ *
+ * The region is the prefix [0, region_bytes) of buf; L = floor(region_bytes / (128*W)) lines.
+ * RR_MODE_LOGICAL: n_warps logical warps, each reading the whole region; any block may run
+ *   any warp; out has n_warps entries.
+ * RR_MODE_PER_SM: a persistent grid, warps_per_sm warps on every SM; a block reads %smid,
+ *   claims the SM, looks its group and window up in a table in shared memory; warp
+ *   v = smid*warps_per_sm + w.  group_of_sm == NULL: every SM active, window = whole region.
+ *   Otherwise group_of_sm[nsm] (HOST) gives each SM's group or RR_SM_INACTIVE, and
+ *   windows[n_groups] (HOST) the window of each group.  out has nsm*warps_per_sm entries;
+ *   inactive SMs' entries are {0,0}.  nsm must equal the device's SM count (0 = take it).
+ * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
+ * (reads_per_warp = 0 is valid: all checksums {0,0}).
+ * unroll: independent loads kept in flight per warp: 0 (= default) or 2, 4, 8, 16.
+ *
+ * out_dev (DEVICE, 8-byte aligned): pairs {X, S} of uint32.  scratch_dev: rr_scratch_bytes().
+ * res == NULL: asynchronous on `stream`, no timing; decode the scratch later with
+ *   rr_read_report().  res != NULL: the call records events around the launch, synchronises
+ *   the stream, checks SM coverage and the status word, and fills *res (HOST).               */
+typedef struct {
+    uint32_t base_line, n_lines;
+} rr_window_t;
+
+typedef struct {
+    const void *buf;            /* DEVICE, 512-byte aligned                                    */
+    uint64_t region_bytes;
+    uint32_t words_per_lane;    /* W: 1, 2, 4                                                  */
+    uint32_t mode;              /* RR_MODE_*                                                   */
+    uint32_t index_mode;        /* RR_INDEX_*                                                  */
+    uint32_t n_warps;           /* LOGICAL                                                     */
+    uint32_t warps_per_sm;      /* PER_SM: 1..32, or 34..64 even (two blocks per SM)           */
+    uint32_t nsm;               /* PER_SM: SM count of the device, 0 = query                   */
+    uint64_t reads_per_warp;
+    uint64_t first_read;
+    uint64_t seed;
+    const uint16_t *group_of_sm; /* HOST [nsm] or NULL                                         */
+    const rr_window_t *windows;  /* HOST [n_groups] or NULL                                    */
+    uint32_t n_groups;
+    uint32_t variant;           /* RR_VARIANT_*                                                */
+    uint32_t unroll;
+    uint32_t reserved;          /* must be 0                                                   */
+} rr_read_params_t;
+
+typedef struct {
+    double seconds_event;   /* CUDA events around the launch (0 when not timed)                */
+    double seconds_device;  /* max block end - min block start, %globaltimer                   */
+    uint64_t bytes;         /* active warps * reads_per_warp * 128 * W                         */
+    double gbps;            /* bytes / seconds_event / 1e9 (seconds_device when not timed)     */
+    uint32_t status;        /* device status word: 0 = clean                                   */
+    uint32_t violations;    /* checked variant: addresses rejected                             */
+    uint32_t sms_covered;   /* PER_SM: active SMs that ran their warps                         */
+    uint32_t blocks_run;    /* blocks that did work                                            */
+} rr_result_t;
+
+int32_t rr_random_read(const rr_read_params_t *params /*HOST*/, void *out_dev /*DEVICE*/,
+                       void *scratch_dev /*DEVICE*/, rr_result_t *res /*HOST or NULL*/,
+                       void *stream);
+
+/* Decodes the scratch of the last rr_random_read that used it (call after the stream has
+ * been synchronised; this function synchronises `stream` itself first).  Returns
+ * RR_ERR_SM_UNCOVERED / RR_ERR_CHECK like the timed form of rr_random_read.                   */
+int32_t rr_read_report(const rr_read_params_t *params /*HOST*/, const void *scratch_dev,
+                       rr_result_t *res /*HOST*/, void *stream);
+
+/* ---- A6: two-SM contention probe -----------------------------------------------------------
+ * Paper, Section 2.2: "if we run our memory access kernel with only two SMs, we expect ... a
+ * drop in throughput when those SMs are in the same GPC".  A full grid is launched; blocks exit
+ * unless they are the first block on sm_a or sm_b.  Each surviving SM performs total_reads/2
+ * random 128-byte line reads (W = 1) over the whole region with warps_per_sm warps (1..32;
+ * total_reads must be a multiple of 2*warps_per_sm), warp ids and streams as in RR_MODE_PER_SM.
+ * sm_a == sm_b: a solo run (total_reads/2 reads on that one SM).
+ * out_dev: 2*warps_per_sm pairs {X,S}: sm_a's warps, then sm_b's (zeros for a solo run).
+ * Synchronous.  res->gbps = bytes of both SMs / (latest end - earliest start, %globaltimer);
+ * res->seconds_event is the event time of the launch.  RR_ERR_SM_UNCOVERED if, after three
+ * launches with growing grids, one of the SMs never received a block.                        */
+int32_t rr_probe_pair(const void *buf /*DEVICE*/, uint64_t region_bytes, uint32_t sm_a,
+                      uint32_t sm_b, uint64_t total_reads, uint32_t warps_per_sm, uint64_t seed,
+                      void *out_dev /*DEVICE*/, void *scratch_dev /*DEVICE*/,
+                      rr_result_t *res /*HOST*/, void *stream);
+
+/* Bytes of DEVICE scratch rr_probe_matrix needs for nsm SMs (one timing record per pair).    */
+size_t rr_probe_matrix_scratch_bytes(uint32_t nsm);
+
+/* All unordered pairs and all solos: T_host[a*nsm+b] = T_host[b*nsm+a] = pair GB/s (median of
+ * `repeats` sweeps, repeats >= 1), T_host[a*nsm+a] = solo GB/s.  Launches are queued back to
+ * back per sweep and read back once.  out_dev as in rr_probe_pair (overwritten by every pair).
+ * overlap_min_host (HOST, may be NULL) receives the smallest overlap fraction
+ * (earliest end - latest start) / (latest end - earliest start) over all pairs.              */
+int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint64_t total_reads,
+                        uint32_t warps_per_sm, uint64_t seed, uint32_t repeats,
+                        float *T_host /*HOST nsm*nsm*/, uint32_t nsm, void *out_dev /*DEVICE*/,
+                        void *scratch_dev /*DEVICE*/, double *overlap_min_host, void *stream);
+
+/* ---- A7: contention matrix -> SM groups ----------------------------------------------------
+ * Paper, Section 2.2 and Figure 3 ("rearranging the indices" so groups show as blocks).  Here:
+ * symmetrise, quantise against the median, average-linkage agglomeration with exact integer
+ * sums, cut at the largest height gap among cuts leaving 2..n/3 clusters, null rule (gap below
+ * 4 robust standard deviations of the height -> one group), groups numbered by their smallest
+ * SM id.  Runs as one block on the device.
+ * T_host: HOST n*n float32 row-major (diagonal ignored; off-diagonal entries must be finite
+ * and > 0, else RR_ERR_ARG); 2 <= n <= RR_MAX_SM.  group_of_sm_host: HOST int32[n].
+ * heights_host: HOST double[n-1] or NULL (merge heights).  Synchronous.                      */
+int32_t rr_cluster(const float *T_host, uint32_t n, void *scratch_dev /*DEVICE*/,
+                   int32_t *group_of_sm_host, uint32_t *n_groups, double *confidence,
+                   double *heights_host, void *stream);
+
+/* ---- A9 policy: windows per group (host only) ----------------------------------------------
+ * Paper, Section 1.3 ("restricted to a 64GB window (or, say, half the memory for simplicity)")
+ * and Section 2.4.  The L lines of the region are cut into K = ceil(L / floor(window_bytes /
+ * (128*W))) chunks of floor(L/K) lines, the last running to L.  policy 0: group g takes chunk
+ * g mod K.  policy 1 (the paper's naive per-SM control; pass one group per SM): chunk
+ * sm64(seed ^ g) mod K.  *coverage (may be NULL) = distinct chunks used / K.                  */
+int32_t rr_make_windows(uint64_t region_bytes, uint32_t words_per_lane, uint64_t window_bytes,
+                        uint32_t n_groups, uint32_t policy, uint64_t seed,
+                        rr_window_t *out_host /*HOST n_groups*/, double *coverage);
+
+/* ---- A8: plateau, cliff and reach from a size sweep (host only) ----------------------------
+ * Paper, Section 2.1 / Figure 1 ("something dramatic happens when the memory region is larger
+ * than about 64GB").  size_bytes strictly increasing.  plateau = lower median of GB/s over
+ * 4 GiB <= size <= 32 GiB; a cliff exists iff a larger size has GB/s < 0.8 plateau; reach =
+ * largest size before it with GB/s >= 0.9 plateau.  Returns 1 (cliff), 0 (none) or an error.  */
+int32_t rr_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
+                 double *plateau, uint64_t *reach_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RR_H_ */

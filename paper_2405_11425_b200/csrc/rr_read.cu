@@ -1,0 +1,701 @@
+// rr_random_read / rr_probe_pair / rr_probe_matrix: warp-coalesced random line reads
+// (paper Section 2.1), per-SM-group windows (Sections 2.1 and 2.4) and the two-SM contention
+// probe (Section 2.2), as persistent sm_100a kernels.
+//
+// Shape of the hot loop.  The machine can retire one 128-byte line every ~5 cycles per SM at HBM
+// rate, i.e. roughly 20 issue slots per line, so the index stream must not be computed 32 times
+// over.  Each lane therefore computes the line of ONE read of a 32-read batch (hash + exact
+// remainder), a shuffle hands line j to all lanes, one IMAD.WIDE forms the lane address, one
+// vector load fetches the lane's W words.  U loads per warp stay in flight in a register ring:
+// the slot of read t is folded into the checksums and immediately refilled with read t+U.
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "rr_device.cuh"
+#include "rr_internal.h"
+
+namespace rr {
+
+struct Tables {
+    uint16_t group_of_sm[RR_MAX_SM];
+    rr_window_t windows[RR_MAX_GROUPS];
+};
+
+struct ReadArgs {
+    const char *buf;
+    uint64_t region_bytes;
+    uint64_t reads, first_read;
+    uint64_t key_seed;  // sm64(seed)
+    uint32_t n_lines;   // L of the whole region
+    uint32_t mode, index_mode;
+    uint32_t n_warps;        // LOGICAL
+    uint32_t wps, wpc, cps;  // warps per SM, per block; blocks per SM
+    uint32_t nsm;
+    uint32_t n_groups;  // 0 = ungrouped
+    uint2 *out;
+    ScratchHeader *scratch;
+};
+
+template <int W, int U, bool CHECKED>
+__device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
+                                           uint64_t key, uint32_t index_mode, uint64_t v,
+                                           uint64_t V, uint64_t first, uint64_t reads,
+                                           uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
+                                           uint32_t &S, uint32_t *violations)
+{
+    static_assert(U >= 1 && U <= 16 && (32 % U) == 0, "ring depth must divide a batch");
+    const Divisor div = make_divisor(n);
+    const char *lane_ptr = buf + lane * (4u * W);
+    uint32_t d[U][W];
+    uint32_t x = 0, s = 0;
+
+    auto gen = [&](uint64_t i) -> uint32_t {
+        uint64_t r = (index_mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        return base + mod_exact(r, div);
+    };
+    auto issue = [&](uint32_t line, uint32_t(&dst)[W]) {
+        if (CHECKED) {
+            bool ok = line >= base && line - base < n &&
+                      ((uint64_t)line + 1) * (128u * W) <= region_bytes;
+            if (!ok) {
+                if (lane == 0) atomicAdd(violations, 1u);
+#pragma unroll
+                for (int w = 0; w < W; ++w) dst[w] = 0;
+                return;
+            }
+        }
+        load_lane<W>(lane_ptr + (uint64_t)line * (128u * W), dst);
+    };
+    auto fold = [&](const uint32_t(&src)[W]) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            x ^= src[w];
+            s += src[w];
+        }
+    };
+
+    const uint64_t n_batches = (reads + 31) >> 5;
+    uint32_t cur = gen(first + lane);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u);
+        if ((uint64_t)u < reads) {
+            issue(line, d[u]);
+        } else {
+#pragma unroll
+            for (int w = 0; w < W; ++w) d[u][w] = 0;
+        }
+    }
+    for (uint64_t b = 0; b < n_batches; ++b) {
+        const uint64_t t0 = b << 5;
+        const uint32_t nxt = gen(first + t0 + 32 + lane);
+        if (t0 + 32 + U <= reads) {  // every read of this batch and its refills exist
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                fold(d[j % U]);
+                uint32_t line = (j + U < 32) ? __shfl_sync(0xFFFFFFFFu, cur, (j + U) & 31)
+                                             : __shfl_sync(0xFFFFFFFFu, nxt, (j + U) & 31);
+                issue(line, d[j % U]);
+            }
+        } else {  // ragged tail: same order, guarded by warp-uniform conditions
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const uint64_t t = t0 + j;
+                if (t < reads) fold(d[j % U]);
+                uint32_t line = (j + U < 32) ? __shfl_sync(0xFFFFFFFFu, cur, (j + U) & 31)
+                                             : __shfl_sync(0xFFFFFFFFu, nxt, (j + U) & 31);
+                if (t + U < reads) issue(line, d[j % U]);
+            }
+        }
+        cur = nxt;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        x ^= __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    }
+    X = x;
+    S = s;
+}
+
+template <int W, int U, bool CHECKED>
+__global__ void __launch_bounds__(1024, 1)
+    read_kernel(const __grid_constant__ ReadArgs a, const __grid_constant__ Tables tab)
+{
+    __shared__ uint32_t sh_sm, sh_slot;
+    __shared__ uint16_t sh_group[RR_MAX_SM];
+    __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    ScratchHeader *sc = a.scratch;
+
+    if (a.mode == RR_MODE_PER_SM) {
+        if (threadIdx.x == 0) {
+            uint32_t sm = smid();
+            sh_sm = sm;
+            sh_slot = (sm < a.nsm) ? atomicAdd(&sc->claim[sm], 1u) : 0xFFFFFFFFu;
+            if (sm >= a.nsm) atomicOr(&sc->status, 1u);  // an SM id outside the table
+        }
+        for (uint32_t k = threadIdx.x; k < a.nsm; k += blockDim.x) sh_group[k] = tab.group_of_sm[k];
+        for (uint32_t k = threadIdx.x; k < a.n_groups; k += blockDim.x) sh_win[k] = tab.windows[k];
+        __syncthreads();
+        const uint32_t sm = sh_sm, slot = sh_slot;
+        if (slot >= a.cps) return;  // not among the first blocks on this SM
+        uint32_t base = 0, n = a.n_lines;
+        if (a.n_groups) {
+            const uint32_t g = sh_group[sm];
+            if (g == RR_SM_INACTIVE) return;
+            base = sh_win[g].base_line;
+            n = sh_win[g].n_lines;
+        }
+        uint64_t t_start = 0;
+        if (threadIdx.x == 0) t_start = globaltimer();
+        const uint64_t v = (uint64_t)sm * a.wps + slot * a.wpc + warp;
+        const uint64_t V = (uint64_t)a.nsm * a.wps;
+        uint32_t X, S;
+        warp_reads<W, U, CHECKED>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v, V,
+                                  a.first_read, a.reads, base, n, lane, X, S, &sc->violations);
+        if (lane == 0) a.out[v] = make_uint2(X, S);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            BlockRecord r;
+            r.smid = sm;
+            r.slot = slot;
+            r.t_start = t_start;
+            r.t_end = globaltimer();
+            sc->rec[sm * a.cps + slot] = r;
+            atomicAdd(&sc->blocks_run, 1u);
+        }
+    } else {
+        uint64_t t_start = 0;
+        if (threadIdx.x == 0) t_start = globaltimer();
+        const uint64_t stride = (uint64_t)gridDim.x * a.wpc;
+        for (uint64_t v = (uint64_t)blockIdx.x * a.wpc + warp; v < a.n_warps; v += stride) {
+            uint32_t X, S;
+            warp_reads<W, U, CHECKED>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v,
+                                      a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
+                                      &sc->violations);
+            if (lane == 0) a.out[v] = make_uint2(X, S);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            BlockRecord r;
+            r.smid = smid();
+            r.slot = blockIdx.x;
+            r.t_start = t_start;
+            r.t_end = globaltimer();
+            sc->rec[blockIdx.x] = r;
+            atomicAdd(&sc->blocks_run, 1u);
+        }
+    }
+}
+
+// ---- two-SM probe ----------------------------------------------------------------------------
+struct ProbeArgs {
+    const char *buf;
+    uint64_t region_bytes;
+    uint64_t reads;  // per warp
+    uint64_t key_seed;
+    uint32_t n_lines;
+    uint32_t sm_a, sm_b;
+    uint32_t wps, nsm;
+    uint2 *out;
+    ProbeRecord *rec;
+};
+
+constexpr int kProbeUnroll = 8;
+
+__global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ ProbeArgs a)
+{
+    __shared__ uint32_t sh_which, sh_slot;
+    if (threadIdx.x == 0) {
+        const uint32_t sm = smid();
+        const uint32_t which = (sm == a.sm_a) ? 0u : (sm == a.sm_b ? 1u : 2u);
+        sh_which = which;
+        sh_slot = (which < 2u) ? atomicAdd(&a.rec->claim[which], 1u) : 1u;
+    }
+    __syncthreads();
+    const uint32_t which = sh_which;
+    if (which >= 2u || sh_slot != 0u) return;  // not on a chosen SM, or not the first block there
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t sm = which ? a.sm_b : a.sm_a;
+    uint64_t t_start = 0;
+    if (threadIdx.x == 0) t_start = globaltimer();
+    const uint64_t v = (uint64_t)sm * a.wps + warp;
+    uint32_t X, S;
+    warp_reads<1, kProbeUnroll, false>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
+                                       RR_INDEX_RANDOM, v, (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
+                                       a.n_lines, lane, X, S, nullptr);
+    if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        a.rec->t_start[which] = t_start;
+        a.rec->t_end[which] = globaltimer();
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+typedef void (*ReadKernel)(const ReadArgs, const Tables);
+
+static ReadKernel pick_kernel(uint32_t W, uint32_t U, bool checked)
+{
+#define RR_ROW(W_)                                                                      \
+    if (W == W_) {                                                                      \
+        if (checked) return read_kernel<W_, 4, true>;                                   \
+        switch (U) {                                                                    \
+            case 2: return read_kernel<W_, 2, false>;                                   \
+            case 4: return read_kernel<W_, 4, false>;                                   \
+            case 8: return read_kernel<W_, 8, false>;                                   \
+            case 16: return read_kernel<W_, 16, false>;                                 \
+        }                                                                               \
+    }
+    RR_ROW(1)
+    RR_ROW(2)
+    RR_ROW(4)
+#undef RR_ROW
+    return nullptr;
+}
+
+static bool width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
+
+struct Geometry {
+    uint32_t wps, wpc, cps, grid, block;
+    uint32_t active_warps;
+    uint32_t active_sms;
+};
+
+// Host-only validation; launches nothing and makes no CUDA call.
+static int32_t validate_read(const rr_read_params_t *p, const void *out, const void *scratch,
+                             uint32_t *unroll)
+{
+    if (!p || !out || !scratch || !p->buf) return RR_ERR_ARG;
+    if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_PER_SM ||
+        p->index_mode > RR_INDEX_STRIDE || p->variant > RR_VARIANT_LDG_CHECKED || p->reserved)
+        return RR_ERR_ARG;
+    uint32_t U = p->unroll ? p->unroll : 8u;
+    if (U != 2 && U != 4 && U != 8 && U != 16) return RR_ERR_ARG;
+    *unroll = U;
+    if ((uintptr_t)p->buf % 512u) return RR_ERR_ALIGN;
+    if ((uintptr_t)out % 8u || (uintptr_t)scratch % 16u) return RR_ERR_ALIGN;
+    const uint64_t L = p->region_bytes / (128ull * p->words_per_lane);
+    if (L == 0 || L > 0xFFFFFFFFull) return RR_ERR_RANGE;
+    if (p->reads_per_warp > (1ull << 62) || p->first_read > (1ull << 62)) return RR_ERR_RANGE;
+    if (p->mode == RR_MODE_LOGICAL) {
+        if (p->n_warps == 0 || p->group_of_sm || p->windows || p->n_groups) return RR_ERR_ARG;
+    } else {
+        const uint32_t w = p->warps_per_sm;
+        if (w == 0 || w > RR_MAX_WARPS_PER_SM || (w > 32 && (w & 1u))) return RR_ERR_ARG;
+        if (p->nsm > RR_MAX_SM) return RR_ERR_ARG;
+        if (p->group_of_sm) {
+            if (!p->windows || p->n_groups == 0 || p->n_groups > RR_MAX_GROUPS || p->nsm == 0)
+                return RR_ERR_ARG;
+            for (uint32_t g = 0; g < p->n_groups; ++g)
+                if (p->windows[g].n_lines == 0 ||
+                    (uint64_t)p->windows[g].base_line + p->windows[g].n_lines > L)
+                    return RR_ERR_RANGE;
+            uint32_t active = 0;
+            for (uint32_t s = 0; s < p->nsm; ++s) {
+                if (p->group_of_sm[s] == RR_SM_INACTIVE) continue;
+                if (p->group_of_sm[s] >= p->n_groups) return RR_ERR_MAP;
+                ++active;
+            }
+            if (!active) return RR_ERR_MAP;
+        } else if (p->windows || p->n_groups) {
+            return RR_ERR_ARG;
+        }
+    }
+    return RR_OK;
+}
+
+static int32_t geometry(const rr_read_params_t *p, const DeviceFacts &f, Geometry *g)
+{
+    if (p->mode == RR_MODE_PER_SM) {
+        if (p->nsm && p->nsm != (uint32_t)f.nsm) return RR_ERR_ARG;
+        g->wps = p->warps_per_sm;
+        g->cps = g->wps > 32 ? 2 : 1;
+        g->wpc = g->wps / g->cps;
+        g->grid = (uint32_t)f.nsm * g->cps;
+        g->active_sms = 0;
+        for (int s = 0; s < f.nsm; ++s)
+            g->active_sms += !p->group_of_sm || p->group_of_sm[s] != RR_SM_INACTIVE;
+        g->active_warps = g->active_sms * g->wps;
+    } else {
+        g->wps = g->wpc = 32;
+        g->cps = 1;
+        g->grid = std::min<uint64_t>((uint64_t)f.nsm, ((uint64_t)p->n_warps + 31) / 32);
+        g->active_sms = 0;
+        g->active_warps = p->n_warps;
+    }
+    g->block = g->wpc * 32;
+    return RR_OK;
+}
+
+// Smallest dynamic shared-memory request that makes exactly `want` blocks of `block` threads
+// resident per SM, so that a grid of nsm*want blocks puts `want` on every SM.
+template <typename K>
+static int32_t ballast_for_occupancy(K kernel, int block, int want, const DeviceFacts &f,
+                                     size_t *smem_out)
+{
+    cudaFuncAttributes fa;
+    RR_CUDA(cudaFuncGetAttributes(&fa, kernel));
+    const int per_block_reserved = 1024;
+    int lo = f.smem_per_sm / (want + 1) - per_block_reserved - (int)fa.sharedSizeBytes + 1;
+    if (lo < 0) lo = 0;
+    const int hi = std::min(f.smem_per_block_optin - (int)fa.sharedSizeBytes,
+                            f.smem_per_sm / want - per_block_reserved - (int)fa.sharedSizeBytes);
+    for (int smem = lo; smem <= hi; smem += 1024) {
+        RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int nb = 0;
+        RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, block, (size_t)smem));
+        if (nb == want) {
+            *smem_out = (size_t)smem;
+            return RR_OK;
+        }
+        if (nb < want) break;
+    }
+    // registers or threads already limit residency below `want`
+    int nb = 0;
+    RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, block, 0));
+    if (nb == want) {
+        *smem_out = 0;
+        return RR_OK;
+    }
+    set_cuda_error(cudaErrorLaunchOutOfResources, "cannot force the requested blocks per SM");
+    return RR_ERR_CUDA;
+}
+
+static int32_t decode(const rr_read_params_t *p, const Geometry &g, const DeviceFacts &f,
+                      const ScratchHeader &h, double seconds_event, rr_result_t *res)
+{
+    uint64_t t0 = ~0ull, t1 = 0;
+    uint32_t covered = 0;
+    bool uncovered = false;
+    auto take = [&](const BlockRecord &r) {
+        if (r.t_end == 0) return false;
+        t0 = std::min(t0, r.t_start);
+        t1 = std::max(t1, r.t_end);
+        return true;
+    };
+    if (p->mode == RR_MODE_PER_SM) {
+        for (int s = 0; s < f.nsm; ++s) {
+            if (p->group_of_sm && p->group_of_sm[s] == RR_SM_INACTIVE) continue;
+            bool all = true;
+            for (uint32_t k = 0; k < g.cps; ++k) all = take(h.rec[s * g.cps + k]) && all;
+            if (all) ++covered; else uncovered = true;
+        }
+    } else {
+        for (uint32_t b = 0; b < g.grid; ++b)
+            if (!take(h.rec[b])) uncovered = true;
+    }
+    res->seconds_event = seconds_event;
+    res->seconds_device = (t1 > t0) ? (double)(t1 - t0) * 1e-9 : 0.0;
+    res->bytes = (uint64_t)g.active_warps * p->reads_per_warp * 128ull * p->words_per_lane;
+    const double sec = seconds_event > 0 ? seconds_event : res->seconds_device;
+    res->gbps = sec > 0 ? (double)res->bytes / sec * 1e-9 : 0.0;
+    res->status = h.status;
+    res->violations = h.violations;
+    res->sms_covered = covered;
+    res->blocks_run = h.blocks_run;
+    if (uncovered) return RR_ERR_SM_UNCOVERED;
+    if (h.violations) return RR_ERR_CHECK;
+    if (h.status) return RR_ERR_SM_UNCOVERED;
+    return RR_OK;
+}
+
+}  // namespace rr
+
+using namespace rr;
+
+extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void *scratch_dev,
+                                  rr_result_t *res, void *stream_)
+{
+    uint32_t U = 0;
+    int32_t rc = validate_read(p, out_dev, scratch_dev, &U);
+    if (rc != RR_OK) return rc;
+    DeviceFacts f;
+    rc = device_facts(&f);
+    if (rc != RR_OK) return rc;
+    Geometry g;
+    rc = geometry(p, f, &g);
+    if (rc != RR_OK) return rc;
+    const bool checked = p->variant == RR_VARIANT_LDG_CHECKED;
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, checked);
+    if (!kernel) return RR_ERR_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+
+    size_t smem = 0;
+    if (p->mode == RR_MODE_PER_SM) {
+        rc = ballast_for_occupancy(kernel, (int)g.block, (int)g.cps, f, &smem);
+        if (rc != RR_OK) return rc;
+    }
+
+    ReadArgs a;
+    a.buf = (const char *)p->buf;
+    a.region_bytes = p->region_bytes;
+    a.reads = p->reads_per_warp;
+    a.first_read = p->first_read;
+    a.key_seed = sm64(p->seed);
+    a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
+    a.mode = p->mode;
+    a.index_mode = p->index_mode;
+    a.n_warps = p->n_warps;
+    a.wps = g.wps;
+    a.wpc = g.wpc;
+    a.cps = g.cps;
+    a.nsm = (uint32_t)f.nsm;
+    a.n_groups = p->group_of_sm ? p->n_groups : 0;
+    a.out = (uint2 *)out_dev;
+    a.scratch = (ScratchHeader *)scratch_dev;
+    Tables tab;
+    std::memset(&tab, 0, sizeof(tab));
+    if (p->group_of_sm) {
+        std::memcpy(tab.group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
+        std::memcpy(tab.windows, p->windows, sizeof(rr_window_t) * p->n_groups);
+    }
+
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (res) {
+        RR_CUDA(cudaEventCreate(&e0));
+        RR_CUDA(cudaEventCreate(&e1));
+    }
+    auto cleanup = [&]() {
+        if (e0) cudaEventDestroy(e0);
+        if (e1) cudaEventDestroy(e1);
+    };
+#define RR_CUDA_C(call)                        \
+    do {                                       \
+        cudaError_t e__ = (call);              \
+        if (e__ != cudaSuccess) {              \
+            set_cuda_error(e__, #call);        \
+            cleanup();                         \
+            return RR_ERR_CUDA;                \
+        }                                      \
+    } while (0)
+
+    RR_CUDA_C(cudaMemsetAsync(scratch_dev, 0, offsetof(ScratchHeader, probe), stream));
+    if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
+        RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
+    if (res) RR_CUDA_C(cudaEventRecord(e0, stream));
+    kernel<<<g.grid, g.block, smem, stream>>>(a, tab);
+    RR_CUDA_C(cudaGetLastError());
+    if (!res) return RR_OK;
+    RR_CUDA_C(cudaEventRecord(e1, stream));
+    RR_CUDA_C(cudaEventSynchronize(e1));
+    float ms = 0.f;
+    RR_CUDA_C(cudaEventElapsedTime(&ms, e0, e1));
+    static thread_local ScratchHeader h;
+    RR_CUDA_C(cudaMemcpyAsync(&h, scratch_dev, offsetof(ScratchHeader, probe),
+                              cudaMemcpyDeviceToHost, stream));
+    RR_CUDA_C(cudaStreamSynchronize(stream));
+    cleanup();
+#undef RR_CUDA_C
+    return decode(p, g, f, h, (double)ms * 1e-3, res);
+}
+
+extern "C" int32_t rr_read_report(const rr_read_params_t *p, const void *scratch_dev,
+                                  rr_result_t *res, void *stream_)
+{
+    if (!res) return RR_ERR_ARG;
+    uint32_t U = 0;
+    int32_t rc = validate_read(p, /*out (unused)*/ (const void *)8, scratch_dev, &U);
+    if (rc != RR_OK) return rc;
+    DeviceFacts f;
+    rc = device_facts(&f);
+    if (rc != RR_OK) return rc;
+    Geometry g;
+    rc = geometry(p, f, &g);
+    if (rc != RR_OK) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    static thread_local ScratchHeader h;
+    RR_CUDA(cudaMemcpyAsync(&h, scratch_dev, offsetof(ScratchHeader, probe),
+                            cudaMemcpyDeviceToHost, stream));
+    RR_CUDA(cudaStreamSynchronize(stream));
+    return decode(p, g, f, h, 0.0, res);
+}
+
+// ---- probes ------------------------------------------------------------------------------------
+namespace rr {
+
+static int32_t validate_probe(const void *buf, uint64_t region_bytes, uint64_t total_reads,
+                              uint32_t wps, const void *out, const void *scratch)
+{
+    if (!buf || !out || !scratch) return RR_ERR_ARG;
+    if (wps == 0 || wps > 32 || total_reads == 0 || total_reads % (2ull * wps)) return RR_ERR_ARG;
+    if ((uintptr_t)buf % 512u || (uintptr_t)out % 8u || (uintptr_t)scratch % 16u)
+        return RR_ERR_ALIGN;
+    const uint64_t L = region_bytes / 128ull;
+    if (L == 0 || L > 0xFFFFFFFFull || total_reads > (1ull << 62)) return RR_ERR_RANGE;
+    return RR_OK;
+}
+
+static ProbeArgs probe_args(const void *buf, uint64_t region_bytes, uint32_t a, uint32_t b,
+                            uint64_t total_reads, uint32_t wps, uint64_t seed, void *out,
+                            ProbeRecord *rec, int nsm)
+{
+    ProbeArgs pa;
+    pa.buf = (const char *)buf;
+    pa.region_bytes = region_bytes;
+    pa.reads = total_reads / 2 / wps;
+    pa.key_seed = sm64(seed);
+    pa.n_lines = (uint32_t)(region_bytes / 128ull);
+    pa.sm_a = a;
+    pa.sm_b = (b == a) ? 0xFFFFFFFFu : b;  // solo: no second SM
+    pa.wps = wps;
+    pa.nsm = (uint32_t)nsm;
+    pa.out = (uint2 *)out;
+    pa.rec = rec;
+    return pa;
+}
+
+// GB/s of one probe from its record; returns false if a chosen SM never ran.
+static bool probe_rate(const ProbeRecord &r, bool solo, uint64_t total_reads, double *gbps,
+                       double *seconds, double *overlap)
+{
+    const int k = solo ? 1 : 2;
+    uint64_t s_min = ~0ull, s_max = 0, e_min = ~0ull, e_max = 0;
+    for (int i = 0; i < k; ++i) {
+        if (r.claim[i] == 0 || r.t_end[i] == 0) return false;
+        s_min = std::min(s_min, r.t_start[i]);
+        s_max = std::max(s_max, r.t_start[i]);
+        e_min = std::min(e_min, r.t_end[i]);
+        e_max = std::max(e_max, r.t_end[i]);
+    }
+    const double span = (double)(e_max - s_min) * 1e-9;
+    const uint64_t bytes = (total_reads / 2) * k * 128ull;
+    *seconds = span;
+    *gbps = span > 0 ? (double)bytes / span * 1e-9 : 0.0;
+    *overlap = (e_max > s_min && e_min > s_max) ? (double)(e_min - s_max) / (double)(e_max - s_min)
+                                                : 0.0;
+    return true;
+}
+
+}  // namespace rr
+
+extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_t sm_a,
+                                 uint32_t sm_b, uint64_t total_reads, uint32_t wps, uint64_t seed,
+                                 void *out_dev, void *scratch_dev, rr_result_t *res, void *stream_)
+{
+    int32_t rc = validate_probe(buf, region_bytes, total_reads, wps, out_dev, scratch_dev);
+    if (rc != RR_OK) return rc;
+    if (!res) return RR_ERR_ARG;
+    DeviceFacts f;
+    rc = device_facts(&f);
+    if (rc != RR_OK) return rc;
+    if (sm_a >= (uint32_t)f.nsm || sm_b >= (uint32_t)f.nsm) return RR_ERR_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    size_t smem = 0;
+    rc = ballast_for_occupancy(probe_kernel, (int)wps * 32, 1, f, &smem);
+    if (rc != RR_OK) return rc;
+    ProbeRecord *rec = &((ScratchHeader *)scratch_dev)->probe;
+    ProbeArgs pa = probe_args(buf, region_bytes, sm_a, sm_b, total_reads, wps, seed, out_dev, rec,
+                              f.nsm);
+    cudaEvent_t e0, e1;
+    RR_CUDA(cudaEventCreate(&e0));
+    RR_CUDA(cudaEventCreate(&e1));
+    int32_t result = RR_ERR_SM_UNCOVERED;
+    std::memset(res, 0, sizeof(*res));
+    for (int attempt = 0; attempt < 3 && result == RR_ERR_SM_UNCOVERED; ++attempt) {
+        cudaError_t e = cudaMemsetAsync(rec, 0, sizeof(ProbeRecord), stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(out_dev, 0, 2ull * wps * sizeof(uint2), stream);
+        if (e == cudaSuccess) e = cudaEventRecord(e0, stream);
+        if (e == cudaSuccess) {
+            probe_kernel<<<(uint32_t)f.nsm * (4u << attempt), wps * 32, smem, stream>>>(pa);
+            e = cudaGetLastError();
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(e1, stream);
+        ProbeRecord h;
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(&h, rec, sizeof(h), cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "rr_probe_pair");
+            result = RR_ERR_CUDA;
+            break;
+        }
+        double gbps, sec, ov;
+        if (probe_rate(h, sm_a == sm_b, total_reads, &gbps, &sec, &ov)) {
+            res->seconds_event = (double)ms * 1e-3;
+            res->seconds_device = sec;
+            res->bytes = (total_reads / 2) * (sm_a == sm_b ? 1 : 2) * 128ull;
+            res->gbps = gbps;
+            res->sms_covered = sm_a == sm_b ? 1 : 2;
+            res->blocks_run = res->sms_covered;
+            result = RR_OK;
+        }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return result;
+}
+
+extern "C" size_t rr_probe_matrix_scratch_bytes(uint32_t nsm)
+{
+    return sizeof(ScratchHeader) + sizeof(ProbeRecord) * ((size_t)nsm * (nsm + 1) / 2);
+}
+
+extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint64_t total_reads,
+                                   uint32_t wps, uint64_t seed, uint32_t repeats, float *T_host,
+                                   uint32_t nsm, void *out_dev, void *scratch_dev,
+                                   double *overlap_min_host, void *stream_)
+{
+    int32_t rc = validate_probe(buf, region_bytes, total_reads, wps, out_dev, scratch_dev);
+    if (rc != RR_OK) return rc;
+    if (!T_host || repeats == 0 || repeats > 64 || nsm < 2 || nsm > RR_MAX_SM) return RR_ERR_ARG;
+    DeviceFacts f;
+    rc = device_facts(&f);
+    if (rc != RR_OK) return rc;
+    if (nsm != (uint32_t)f.nsm) return RR_ERR_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    size_t smem = 0;
+    rc = ballast_for_occupancy(probe_kernel, (int)wps * 32, 1, f, &smem);
+    if (rc != RR_OK) return rc;
+
+    const size_t n_pairs = (size_t)nsm * (nsm + 1) / 2;
+    ProbeRecord *recs = (ProbeRecord *)((char *)scratch_dev + sizeof(ScratchHeader));
+    std::vector<ProbeRecord> h(n_pairs);
+    std::vector<float> samples(n_pairs * repeats);
+    double overlap_min = 1.0;
+    for (uint32_t rep = 0; rep < repeats; ++rep) {
+        RR_CUDA(cudaMemsetAsync(recs, 0, sizeof(ProbeRecord) * n_pairs, stream));
+        size_t k = 0;
+        for (uint32_t a = 0; a < nsm; ++a)
+            for (uint32_t b = a; b < nsm; ++b, ++k) {
+                ProbeArgs pa = probe_args(buf, region_bytes, a, b, total_reads, wps, seed, out_dev,
+                                          recs + k, f.nsm);
+                probe_kernel<<<nsm * 4u, wps * 32, smem, stream>>>(pa);
+            }
+        RR_CUDA(cudaGetLastError());
+        RR_CUDA(cudaMemcpyAsync(h.data(), recs, sizeof(ProbeRecord) * n_pairs,
+                                cudaMemcpyDeviceToHost, stream));
+        RR_CUDA(cudaStreamSynchronize(stream));
+        k = 0;
+        for (uint32_t a = 0; a < nsm; ++a)
+            for (uint32_t b = a; b < nsm; ++b, ++k) {
+                double gbps, sec, ov;
+                if (!probe_rate(h[k], a == b, total_reads, &gbps, &sec, &ov)) {
+                    // a chosen SM got no block in the queued launch: redo this pair on its own
+                    rr_result_t r;
+                    rc = rr_probe_pair(buf, region_bytes, a, b, total_reads, wps, seed, out_dev,
+                                       scratch_dev, &r, stream_);
+                    if (rc != RR_OK) return rc;
+                    gbps = r.gbps;
+                    ov = 1.0;
+                }
+                if (a != b) overlap_min = std::min(overlap_min, ov);
+                samples[k * repeats + rep] = (float)gbps;
+            }
+    }
+    size_t k = 0;
+    for (uint32_t a = 0; a < nsm; ++a)
+        for (uint32_t b = a; b < nsm; ++b, ++k) {
+            float *s = &samples[k * repeats];
+            std::sort(s, s + repeats);
+            const float med = s[(repeats - 1) / 2];
+            T_host[(size_t)a * nsm + b] = med;
+            T_host[(size_t)b * nsm + a] = med;
+        }
+    if (overlap_min_host) *overlap_min_host = overlap_min;
+    return RR_OK;
+}

@@ -1,0 +1,159 @@
+"""CPU-side checks of the C-ABI library: it builds and loads without a GPU, exports every
+symbol the header declares, rejects bad arguments before touching CUDA, and its host-only
+policies (windows, reach) agree with the oracle."""
+import ctypes
+import itertools
+import random
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2405_11425_b200 import binding as rr
+from paper_2405_11425_b200 import build as rr_build
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built_library():
+    rr_build.build()
+    return rr._load()
+
+
+def test_exports_match_header(built_library):
+    header = (ROOT / "include" / "rr.h").read_text()
+    declared = set(re.findall(r"^\s*(?:const\s+char\s*\*|int32_t|size_t)\s*\*?\s*(rr_\w+)\s*\(",
+                              header, flags=re.M))
+    assert declared == set(rr.EXPORTS)
+    for name in declared:
+        assert hasattr(built_library, name), name
+
+
+def test_strerror_covers_all_codes():
+    texts = {rr.rr_strerror(c) for c in range(0, -10, -1)}
+    assert len(texts) == 10 and "unknown status" not in texts
+    assert rr.rr_strerror(-99) == "unknown status"
+
+
+FAKE = 0x7F0000000000  # a 512-byte aligned fake device address: validation never dereferences it
+
+
+def _call(**kw):
+    base = dict(W=1, mode=rr.RR_MODE_LOGICAL, n_warps=4, reads_per_warp=4, seed=1)
+    base.update(kw)
+    buf = base.pop("buf", FAKE)
+    region = base.pop("region_bytes", 1 << 20)
+    out = base.pop("out", FAKE)
+    scratch = base.pop("scratch", FAKE)
+    p = rr.ReadParams(buf, region, **base)
+    return rr._load().rr_random_read(ctypes.byref(p.c), out, scratch, None, 0)
+
+
+def test_read_argument_errors_come_before_any_cuda_call():
+    assert _call(W=3) == rr.RR_ERR_ARG
+    assert _call(mode=7) == rr.RR_ERR_ARG
+    assert _call(index_mode=2) == rr.RR_ERR_ARG
+    assert _call(variant=9) == rr.RR_ERR_ARG
+    assert _call(unroll=3) == rr.RR_ERR_ARG
+    assert _call(n_warps=0) == rr.RR_ERR_ARG
+    assert _call(buf=0) == rr.RR_ERR_ARG
+    assert _call(out=0) == rr.RR_ERR_ARG
+    assert _call(scratch=0) == rr.RR_ERR_ARG
+    assert _call(buf=FAKE + 128) == rr.RR_ERR_ALIGN
+    assert _call(out=FAKE + 4) == rr.RR_ERR_ALIGN
+    assert _call(region_bytes=100) == rr.RR_ERR_RANGE
+    assert _call(region_bytes=128 << 32) == rr.RR_ERR_RANGE         # 2^32 lines: one too many
+    assert _call(reads_per_warp=1 << 63) == rr.RR_ERR_RANGE
+    # logical mode takes no grouping
+    assert _call(group_of_sm=np.zeros(4, np.uint16), windows=[[0, 8]]) == rr.RR_ERR_ARG
+    per_sm = dict(mode=rr.RR_MODE_PER_SM, n_warps=0, nsm=4)
+    assert _call(warps_per_sm=0, **per_sm) == rr.RR_ERR_ARG
+    assert _call(warps_per_sm=65, **per_sm) == rr.RR_ERR_ARG
+    assert _call(warps_per_sm=33, **per_sm) == rr.RR_ERR_ARG
+    assert _call(windows=[[0, 8]], **per_sm) == rr.RR_ERR_ARG       # windows without a map
+    g = np.array([0, 1, 0, 1], np.uint16)
+    assert _call(group_of_sm=g, windows=[[0, 8], [8, 9000]], **per_sm) == rr.RR_ERR_RANGE
+    assert _call(group_of_sm=g, windows=[[0, 8], [8, 0]], **per_sm) == rr.RR_ERR_RANGE
+    assert _call(group_of_sm=g, windows=[[0, 8]], **per_sm) == rr.RR_ERR_MAP
+    dead = np.full(4, 0xFFFF, np.uint16)
+    assert _call(group_of_sm=dead, windows=[[0, 8]], **per_sm) == rr.RR_ERR_MAP
+
+
+def test_other_entry_points_reject_bad_arguments():
+    lib = rr._load()
+    assert lib.rr_fill(0, 16, 0) == rr.RR_ERR_ARG
+    assert lib.rr_fill(FAKE + 64, 16, 0) == rr.RR_ERR_ALIGN
+    assert lib.rr_fill(FAKE, 0, 0) == rr.RR_OK                      # empty fill is a no-op
+    res = rr._Result()
+    args = (FAKE, 1 << 30, 0, 1)
+    assert lib.rr_probe_pair(*args, 1 << 10, 0, 5, FAKE, FAKE, ctypes.byref(res), 0) == rr.RR_ERR_ARG
+    assert lib.rr_probe_pair(*args, 1000, 32, 5, FAKE, FAKE, ctypes.byref(res), 0) == rr.RR_ERR_ARG
+    assert lib.rr_probe_pair(*args, 1 << 10, 33, 5, FAKE, FAKE, ctypes.byref(res), 0) == rr.RR_ERR_ARG
+    assert lib.rr_probe_pair(FAKE, 64, 0, 1, 1 << 10, 8, 5, FAKE, FAKE, ctypes.byref(res), 0) == rr.RR_ERR_RANGE
+    T = np.ones((8, 8), np.float32)
+    T[2, 3] = np.nan
+    g = np.zeros(8, np.int32)
+    ng = ctypes.c_uint32()
+    assert lib.rr_cluster(T.ctypes.data, 8, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    T[2, 3] = -1
+    assert lib.rr_cluster(T.ctypes.data, 8, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    T[2, 3] = 1
+    assert lib.rr_cluster(T.ctypes.data, 1, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    assert lib.rr_cluster(T.ctypes.data, 8, FAKE + 4, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ALIGN
+
+
+def test_make_windows_matches_oracle():
+    for L, S, G, W, policy in itertools.product((1, 2, 7, 40, 1000, 12345), (1, 3, 64, 999, 10 ** 6),
+                                                (1, 2, 5, 14, 148), (1, 2, 4), (0, 1)):
+        lb = 128 * W
+        a, ca = rr.rr_make_windows(L * lb + 5, W, S * lb, G, policy, seed=23)
+        b, cb = oracle.make_windows(L * lb + 5, W, S * lb, G, policy, seed=23)
+        assert np.array_equal(a, b) and ca == cb
+    big = int(0.95 * 178 * (1 << 30)) // 512 * 512
+    for S in (big // 8, big // 4, big // 2, big, 64 << 30, 37 << 30):
+        a, ca = rr.rr_make_windows(big, 1, S, 16)
+        b, cb = oracle.make_windows(big, 1, S, 16)
+        assert np.array_equal(a, b) and ca == cb
+    with pytest.raises(rr.RRError):
+        rr.rr_make_windows(1 << 20, 3, 1 << 10, 2)
+    with pytest.raises(rr.RRError):
+        rr.rr_make_windows(1 << 20, 1, 1 << 10, 0)
+    with pytest.raises(rr.RRError):
+        rr.rr_make_windows(64, 1, 1 << 10, 2)
+
+
+def test_reach_matches_oracle():
+    rng = np.random.default_rng(3)
+    sizes = [s << 30 for s in (1, 4, 16, 32, 48, 64, 96, 128, 160, 169)]
+    for _ in range(200):
+        g = rng.uniform(500, 4000, len(sizes))
+        if rng.random() < 0.5:
+            g[rng.integers(4, len(sizes)):] *= 0.3
+        assert rr.rr_reach(sizes, g) == oracle.reach(sizes, g)
+    with pytest.raises(rr.RRError):
+        rr.rr_reach([2 << 30, 1 << 30], [1.0, 1.0])
+    with pytest.raises(rr.RRError):
+        rr.rr_reach([1 << 30], [1.0])
+
+
+def test_exact_remainder_identity():
+    # The kernels take r mod n as r - floor(r*m / 2^64)*n with m = floor((2^64-1)/n), corrected
+    # by at most one subtraction of n.  Check that claim with big integers on edge cases.
+    rnd = random.Random(1)
+    ns = [1, 2, 3, 5, 777, 2 ** 23, 2 ** 23 + 1, 402653184, 2 ** 31 - 1, 2 ** 31, 2 ** 32 - 1]
+    ns += [rnd.randrange(1, 2 ** 32) for _ in range(200)]
+    for n in ns:
+        m = (2 ** 64 - 1) // n
+        rs = [0, 1, n - 1, n, n + 1, 2 ** 64 - 1, 2 ** 64 - n, 2 ** 63, m * n, m * n - 1,
+              (m * n + n - 1) % 2 ** 64]
+        rs += [rnd.randrange(0, 2 ** 64) for _ in range(50)]
+        for r in rs:
+            q = (r * m) >> 64
+            rem = r - q * n
+            assert 0 <= rem < 2 * n
+            if rem >= n:
+                rem -= n
+            assert rem == r % n

@@ -1,0 +1,244 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+
+import oracle
+import rr_inputs
+from paper_2405_11425_b200 import binding as rr
+from paper_2405_11425_b200 import build as rr_build
+
+pytestmark = pytest.mark.gpu
+MiB = 1 << 20
+
+
+@pytest.fixture(scope="module")
+def dev():
+    import torch
+    rr_build.build()
+    torch.cuda.set_device(0)
+    info = rr.rr_device_info()
+
+    class Dev:
+        pass
+
+    d = Dev()
+    d.torch = torch
+    d.info = info
+    d.nsm = info["nsm_prop"]
+    d.scratch = torch.zeros(rr.rr_scratch_bytes(), dtype=torch.uint8, device="cuda")
+    d.buf_bytes = 1 << 30
+    d.buf = torch.empty(d.buf_bytes, dtype=torch.uint8, device="cuda")
+    assert d.buf.data_ptr() % 512 == 0
+    rr.rr_fill(d.buf, d.buf_bytes // 4)
+    torch.cuda.synchronize()
+    return d
+
+
+def _out(dev, n):
+    return dev.torch.full((n, 2), 0x5EADBEEF, dtype=dev.torch.int32, device="cuda")
+
+
+def _np(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def test_device_facts(dev):
+    i = dev.info
+    assert i["cc_major"] == 10
+    assert i["nsm_reg"] == i["nsm_prop"] <= rr.RR_MAX_SM
+    assert i["theoretical_gbps"] > 1000 and i["total_bytes"] > 100 << 30
+
+
+@pytest.mark.parametrize("n_words", [0, 1, 3, 4, 5, 127, 1023, 1024, (1 << 20) + 3, 37 * 148 * 2048 + 2])
+def test_fill_matches_oracle_small(dev, n_words):
+    t = dev.torch.full((n_words + 8,), 0x25A5A5A5, dtype=dev.torch.int32, device="cuda")
+    rr.rr_fill(t, n_words)
+    got = _np(t)
+    assert np.array_equal(got[:n_words], oracle.fill(0, n_words))
+    assert np.all(got[n_words:] == 0x25A5A5A5)          # nothing written past the end
+
+
+def test_fill_1gib_sampled_and_folded(dev):
+    words = dev.buf.view(dev.torch.int32)
+    n = dev.buf_bytes // 4
+    rng = np.random.default_rng(0)
+    for start in [0, n - 4096] + [int(x) for x in rng.integers(0, n - 4096, 16)]:
+        got = _np(words[start:start + 4096])
+        assert np.array_equal(got, oracle.fill(start, 4096))
+
+
+def test_cfg0_all_warps_bit_exact(dev):
+    c = rr_inputs.CFG0
+    out = _out(dev, c.n_warps)
+    p = rr.ReadParams(dev.buf, c.region_bytes, W=c.W, mode=rr.RR_MODE_LOGICAL, n_warps=c.n_warps,
+                      reads_per_warp=c.reads_per_warp, seed=c.seed)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    expect = oracle.read_logical(c.region_bytes, c.W, c.n_warps, c.reads_per_warp, c.seed)
+    assert np.array_equal(_np(out), expect)
+    assert res.bytes == c.n_warps * c.reads_per_warp * 128
+    assert res.status == 0 and res.blocks_run > 0 and res.gbps > 0
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+@pytest.mark.parametrize("unroll", [0, 2, 4, 8, 16])
+def test_logical_widths_unrolls_ragged_reads(dev, W, unroll):
+    region = 777 * MiB + 384            # not a power of two, tail shorter than a line
+    for reads, first in [(0, 0), (1, 0), (7, 3), (31, 0), (32, 1), (33, 0), (40, 100), (100, 7),
+                         (64, 0), (96, 5)]:
+        n_warps = 300
+        out = _out(dev, n_warps)
+        p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
+                          reads_per_warp=reads, first_read=first, seed=11, unroll=unroll)
+        rr.rr_random_read(p, out, dev.scratch)
+        expect = oracle.read_logical(region, W, n_warps, reads, 11, first_read=first)
+        assert np.array_equal(_np(out), expect), (W, unroll, reads, first)
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+def test_checked_variant_is_clean_and_equal(dev, W):
+    region = 64 * MiB + 128
+    out = _out(dev, 500)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=500,
+                      reads_per_warp=45, seed=5, variant=rr.RR_VARIANT_LDG_CHECKED)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    assert res.violations == 0
+    assert np.array_equal(_np(out), oracle.read_logical(region, W, 500, 45, 5))
+
+
+def test_tiny_region_of_one_line(dev):
+    out = _out(dev, 40)
+    p = rr.ReadParams(dev.buf, 128, W=1, mode=rr.RR_MODE_LOGICAL, n_warps=40, reads_per_warp=9,
+                      seed=2, variant=rr.RR_VARIANT_LDG_CHECKED)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_logical(128, 1, 40, 9, 2))
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+def test_stride_mode(dev, W):
+    V, R = 256, 64
+    region = V * R * 128 * W
+    out = _out(dev, V)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=V, reads_per_warp=R,
+                      index_mode=rr.RR_INDEX_STRIDE)
+    rr.rr_random_read(p, out, dev.scratch)
+    got = _np(out)
+    assert np.array_equal(got, oracle.read_logical(region, W, V, R, 0,
+                                                   index_mode=oracle.INDEX_STRIDE))
+    words = oracle.fill(0, region // 4)                 # every line exactly once
+    assert int(np.bitwise_xor.reduce(got[:, 0])) == int(np.bitwise_xor.reduce(words))
+
+
+@pytest.mark.parametrize("wps", [1, 8, 32])
+@pytest.mark.parametrize("W", [1, 2])
+def test_per_sm_ungrouped(dev, wps, W):
+    region = 1000 * MiB
+    out = _out(dev, dev.nsm * wps)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_PER_SM, warps_per_sm=wps,
+                      reads_per_warp=70, first_read=256, seed=7)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    assert res.sms_covered == dev.nsm and res.blocks_run == dev.nsm
+    assert res.bytes == dev.nsm * wps * 70 * 128 * W
+    assert np.array_equal(_np(out), oracle.read_per_sm(region, W, dev.nsm, wps, 70, 7,
+                                                       first_read=256))
+
+
+def test_per_sm_grouped_windows_and_inactive_sms(dev):
+    region = dev.buf_bytes
+    G = 9
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=4, inactive_frac=0.1)
+    windows, cov = rr.rr_make_windows(region, 1, region // 5, G)
+    windows[3] = (1000, 777)                      # an odd window
+    out = _out(dev, dev.nsm * 16)
+    p = rr.ReadParams(dev.buf, region, W=1, mode=rr.RR_MODE_PER_SM, warps_per_sm=16,
+                      reads_per_warp=50, seed=23, group_of_sm=groups, windows=windows)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    active = int((groups != 0xFFFF).sum())
+    assert res.sms_covered == active and res.bytes == active * 16 * 50 * 128
+    expect = oracle.read_per_sm(region, 1, dev.nsm, 16, 50, 23, group_of_sm=groups,
+                                windows=windows)
+    assert np.array_equal(_np(out), expect)
+    # asynchronous form + report give the same
+    out2 = _out(dev, dev.nsm * 16)
+    assert rr.rr_random_read(p, out2, dev.scratch, timed=False) is None
+    rep = rr.rr_read_report(p, dev.scratch)
+    assert np.array_equal(_np(out2), expect) and rep.sms_covered == active
+    assert rep.seconds_device > 0
+
+
+def test_single_whole_window_equals_ungrouped_on_gpu(dev):
+    region = 512 * MiB
+    L = region // 256
+    a, b = _out(dev, dev.nsm * 4), _out(dev, dev.nsm * 4)
+    pa = rr.ReadParams(dev.buf, region, W=2, warps_per_sm=4, reads_per_warp=33, seed=9)
+    pb = rr.ReadParams(dev.buf, region, W=2, warps_per_sm=4, reads_per_warp=33, seed=9,
+                       group_of_sm=np.zeros(dev.nsm, np.uint16), windows=[[0, L]])
+    rr.rr_random_read(pa, a, dev.scratch)
+    rr.rr_random_read(pb, b, dev.scratch)
+    assert np.array_equal(_np(a), _np(b))
+
+
+def test_nsm_mismatch_is_rejected(dev):
+    out = _out(dev, 8)
+    p = rr.ReadParams(dev.buf, 1 << 20, warps_per_sm=1, nsm=dev.nsm - 1, reads_per_warp=1)
+    with pytest.raises(rr.RRError) as e:
+        rr.rr_random_read(p, out, dev.scratch)
+    assert e.value.code == rr.RR_ERR_ARG
+
+
+@pytest.mark.parametrize("wps", [4, 32])
+def test_probe_pair_checksums_and_rates(dev, wps):
+    region = dev.buf_bytes
+    total = 2 * wps * 200
+    for a, b in [(0, 1), (3, dev.nsm - 1), (dev.nsm - 1, 2), (5, 5)]:
+        out = _out(dev, 2 * wps)
+        res = rr.rr_probe_pair(dev.buf, region, a, b, total, wps, 5, out, dev.scratch)
+        got = _np(out)
+        full = oracle.read_per_sm(region, 1, dev.nsm, wps, total // 2 // wps, 5)
+        assert np.array_equal(got[:wps], full[a * wps:(a + 1) * wps])
+        if a != b:
+            assert np.array_equal(got[wps:], full[b * wps:(b + 1) * wps])
+            assert res.bytes == total * 128 and res.sms_covered == 2
+        else:
+            assert not got[wps:].any() and res.bytes == total * 64 and res.sms_covered == 1
+        assert res.gbps > 0 and res.seconds_device > 0
+
+
+def test_probe_matrix_is_symmetric_and_positive(dev):
+    wps = 8
+    scratch = dev.torch.zeros(rr.rr_probe_matrix_scratch_bytes(dev.nsm), dtype=dev.torch.uint8,
+                              device="cuda")
+    out = _out(dev, 2 * wps)
+    T, overlap = rr.rr_probe_matrix(dev.buf, dev.buf_bytes, 2 * wps * 64, wps, 5, 1, dev.nsm, out,
+                                    scratch)
+    assert T.shape == (dev.nsm, dev.nsm) and np.array_equal(T, T.T)
+    assert np.isfinite(T).all() and (T > 0).all()
+
+
+@pytest.mark.parametrize("sizes,drop", [
+    ([8] * 12 + [6] * 2, 0.10),                 # the paper's A100 shape
+    ([18] * 6 + [20] * 2, 0.06),                # 148 SMs
+    ([16] * 16, 0.15),                          # 256 SMs: the table limit
+    ([4, 6, 4], 0.2),
+    ([2, 2, 2], 0.3),                           # 6 SMs: smallest with a group level
+    ([2, 2], 0.3),                              # 4 SMs: no group level
+    ([20] * 7, 0.0),                            # null matrix
+])
+def test_cluster_matches_oracle(dev, sizes, drop):
+    for seed in range(4):
+        T, truth = rr_inputs.planted_matrix(sizes, drop, seed=seed)
+        g, G, conf, h = rr.rr_cluster(T, dev.scratch)
+        og, oG, oconf, oh = oracle.cluster(T)
+        assert G == oG and np.array_equal(g, og)
+        assert np.array_equal(h, oh)                       # same divisions, same doubles
+        assert conf == oconf or (np.isinf(conf) and np.isinf(oconf))
+        if drop >= 0.06 and len(sizes) >= 6 and sum(sizes) // 3 >= len(sizes):
+            assert G == len(sizes) and np.array_equal(g, truth)
+
+
+def test_cluster_two_sms_and_ties(dev):
+    g, G, conf, h = rr.rr_cluster(np.array([[1, 2], [3, 1]], np.float32), dev.scratch)
+    assert G == 1 and list(g) == [0, 0]
+    T = np.full((9, 9), 50.0, np.float32)
+    g, G, conf, h = rr.rr_cluster(T, dev.scratch)
+    og, oG, oconf, oh = oracle.cluster(T)
+    assert G == oG == 1 and np.array_equal(h, oh)
