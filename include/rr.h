@@ -199,10 +199,14 @@ int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint6
  * sums, cut at the largest height gap among cuts leaving 2..n/3 clusters, null rule (gap below
  * 4 robust standard deviations of the height -> one group), groups numbered by their smallest
  * SM id.  Runs as one block on the device.
- * T_host: HOST n*n float32 row-major (diagonal ignored; off-diagonal entries must be finite
- * and > 0, else RR_ERR_ARG); 2 <= n <= RR_MAX_SM.  group_of_sm_host: HOST int32[n].
+ * T_host: HOST n*n float32 row-major; off-diagonal entries must be finite and > 0, else
+ * RR_ERR_ARG; 2 <= n <= RR_MAX_SM.  flags = 0: the diagonal is ignored.
+ * flags = RR_CLUSTER_SOLO_NORMALISE: every pair entry is first divided by the sum of the two
+ * SMs' solo rates on the diagonal (which must then be finite and > 0), so an SM that is slow
+ * on its own does not look contended.  group_of_sm_host: HOST int32[n].
  * heights_host: HOST double[n-1] or NULL (merge heights).  Synchronous.                      */
-int32_t rr_cluster(const float *T_host, uint32_t n, void *scratch_dev /*DEVICE*/,
+#define RR_CLUSTER_SOLO_NORMALISE 1u
+int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratch_dev /*DEVICE*/,
                    int32_t *group_of_sm_host, uint32_t *n_groups, double *confidence,
                    double *heights_host, void *stream);
 

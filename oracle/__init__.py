@@ -68,7 +68,7 @@ def _load():
         lib.orc_make_windows.restype = i32
         lib.orc_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p, p]
         lib.orc_cluster.restype = i32
-        lib.orc_cluster.argtypes = [p, u32, p, p, p, p]
+        lib.orc_cluster.argtypes = [p, u32, u32, p, p, p, p]
         lib.orc_reach.restype = i32
         lib.orc_reach.argtypes = [p, p, u32, p, p]
         _lib = lib
@@ -169,8 +169,10 @@ def make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int, po
     return np.stack([wb, wn], axis=1), float(cov.value)
 
 
-def cluster(T):
-    """SM x SM throughput matrix -> (group_of_sm int32[n], n_groups, confidence, heights[n-1])."""
+def cluster(T, solo_normalise: bool = False):
+    """SM x SM throughput matrix -> (group_of_sm int32[n], n_groups, confidence, heights[n-1]).
+
+    ``solo_normalise`` divides every pair entry by the sum of the two solo rates on the diagonal."""
     T = np.ascontiguousarray(T, dtype=np.float32)
     n = T.shape[0]
     if T.shape != (n, n):
@@ -179,7 +181,7 @@ def cluster(T):
     heights = np.zeros(max(n - 1, 1), dtype=np.float64)
     ng = ctypes.c_uint32()
     conf = ctypes.c_double()
-    rc = _load().orc_cluster(_ptr(T), n, _ptr(groups), ctypes.byref(ng), ctypes.byref(conf),
+    rc = _load().orc_cluster(_ptr(T), n, 1 if solo_normalise else 0, _ptr(groups), ctypes.byref(ng), ctypes.byref(conf),
                              _ptr(heights))
     if rc != 0:
         raise OracleError(rc)

@@ -216,7 +216,10 @@ int32_t orc_make_windows(uint64_t region_bytes, uint32_t W, uint64_t window_byte
 }
 
 /* ---- O5: SM x SM matrix -> groups (Section 2.2, Figures 2 and 3) ---------------
- * 1. symmetrise off-diagonal entries in double: t = (T_ij + T_ji) / 2
+ * 1. symmetrise off-diagonal entries in double: t = (T_ij + T_ji) / 2; with flag
+ *    ORC_CLUSTER_SOLO_NORMALISE, divide by the two SMs' solo rates on the diagonal:
+ *    t = t / (T_ii + T_jj), so that an SM that is slower on its own is not mistaken
+ *    for a contended one (1.0 = the pair runs as fast as the two solos together)
  * 2. quantise: q = rint(t * 2^20 / lower-median(t)), clamped to 2^32-1
  * 3. average linkage on q (small q = contended = close): exact integer pair sums,
  *    means compared by cross-multiplication, ties -> smallest (a,b); a cluster is
@@ -239,10 +242,12 @@ static int cmp_u32(const void *a, const void *b)
     return (x > y) - (x < y);
 }
 
-int32_t orc_cluster(const float *T, uint32_t n, int32_t *group_of_sm, uint32_t *n_groups,
-                    double *confidence, double *heights)
+#define ORC_CLUSTER_SOLO_NORMALISE 1u
+
+int32_t orc_cluster(const float *T, uint32_t n, uint32_t flags, int32_t *group_of_sm,
+                    uint32_t *n_groups, double *confidence, double *heights)
 {
-    if (!T || !group_of_sm || !n_groups || n < 2 || n > 256) return ORC_ERR_ARG;
+    if (!T || !group_of_sm || !n_groups || n < 2 || n > 256 || flags > 1) return ORC_ERR_ARG;
     size_t m = (size_t)n * (n - 1) / 2;
     double *t = (double *)malloc(sizeof(double) * (size_t)n * n);
     double *sorted = (double *)malloc(sizeof(double) * m);
@@ -273,6 +278,14 @@ int32_t orc_cluster(const float *T, uint32_t n, int32_t *group_of_sm, uint32_t *
                     goto done;
                 }
                 double s = (a + b) * 0.5;
+                if (flags & ORC_CLUSTER_SOLO_NORMALISE) {
+                    double di = (double)T[(size_t)i * n + i], dj = (double)T[(size_t)j * n + j];
+                    if (!(di > 0.0) || !(dj > 0.0) || isinf(di) || isinf(dj)) {
+                        rc = ORC_ERR_ARG;
+                        goto done;
+                    }
+                    s = s / (di + dj);
+                }
                 t[(size_t)i * n + j] = s;
                 t[(size_t)j * n + i] = s;
                 sorted[k++] = s;

@@ -128,7 +128,7 @@ def _load():
     lib.rr_probe_matrix.restype = i32
     lib.rr_probe_matrix.argtypes = [p, u64, u64, u32, u64, u32, p, u32, p, p, p, p]
     lib.rr_cluster.restype = i32
-    lib.rr_cluster.argtypes = [p, u32, p, p, p, p, p, p]
+    lib.rr_cluster.argtypes = [p, u32, u32, p, p, p, p, p, p]
     lib.rr_make_windows.restype = i32
     lib.rr_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p]
     lib.rr_reach.restype = i32
@@ -250,7 +250,10 @@ def rr_probe_matrix(buf, region_bytes: int, total_reads: int, warps_per_sm: int,
     return T, float(ov.value)
 
 
-def rr_cluster(T, scratch, stream=None):
+RR_CLUSTER_SOLO_NORMALISE = 1
+
+
+def rr_cluster(T, scratch, flags: int = 0, stream=None):
     """Returns (group_of_sm int32[n], n_groups, confidence, heights float64[n-1])."""
     T = np.ascontiguousarray(T, dtype=np.float32)
     n = int(T.shape[0])
@@ -260,7 +263,7 @@ def rr_cluster(T, scratch, stream=None):
     heights = np.zeros(max(n - 1, 1), dtype=np.float64)
     ng = ctypes.c_uint32()
     conf = ctypes.c_double()
-    _check(_load().rr_cluster(T.ctypes.data, n, _dev(scratch), groups.ctypes.data,
+    _check(_load().rr_cluster(T.ctypes.data, n, flags, _dev(scratch), groups.ctypes.data,
                               ctypes.byref(ng), ctypes.byref(conf), heights.ctypes.data,
                               _stream(stream)), "rr_cluster")
     return groups, int(ng.value), float(conf.value), heights[: n - 1]

@@ -93,7 +93,7 @@ __device__ __forceinline__ Candidate shfl_down(const Candidate &c, int o)
     return r;
 }
 
-__global__ void __launch_bounds__(kClusterThreads, 1) cluster_kernel(uint8_t *work, uint32_t n)
+__global__ void __launch_bounds__(kClusterThreads, 1) cluster_kernel(uint8_t *work, uint32_t n, uint32_t flags)
 {
     const ClusterLayout lay(n);
     const float *T = (const float *)(work + lay.off_T);
@@ -114,7 +114,10 @@ __global__ void __launch_bounds__(kClusterThreads, 1) cluster_kernel(uint8_t *wo
 
     // 1. symmetrised off-diagonal entries, as sortable keys (positive doubles order like integers)
     auto sym = [&](uint32_t i, uint32_t j) {
-        return __dmul_rn(__dadd_rn((double)T[i * n + j], (double)T[j * n + i]), 0.5);
+        double s = __dmul_rn(__dadd_rn((double)T[i * n + j], (double)T[j * n + i]), 0.5);
+        if (flags & RR_CLUSTER_SOLO_NORMALISE)  // pair rate relative to the two solo rates
+            s = __ddiv_rn(s, __dadd_rn((double)T[i * n + i], (double)T[j * n + j]));
+        return s;
     };
     for (uint32_t k = tid; k < lay.pow2; k += blockDim.x) keys[k] = ~0ull;
     __syncthreads();
@@ -280,17 +283,18 @@ __global__ void __launch_bounds__(kClusterThreads, 1) cluster_kernel(uint8_t *wo
 
 using namespace rr;
 
-extern "C" int32_t rr_cluster(const float *T_host, uint32_t n, void *scratch_dev,
+extern "C" int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratch_dev,
                               int32_t *group_of_sm_host, uint32_t *n_groups, double *confidence,
                               double *heights_host, void *stream_)
 {
-    if (!T_host || !scratch_dev || !group_of_sm_host || !n_groups || n < 2 || n > RR_MAX_SM)
+    if (!T_host || !scratch_dev || !group_of_sm_host || !n_groups || n < 2 || n > RR_MAX_SM ||
+        flags > RR_CLUSTER_SOLO_NORMALISE)
         return RR_ERR_ARG;
     if ((uintptr_t)scratch_dev % 16u) return RR_ERR_ALIGN;
     for (uint32_t i = 0; i < n; ++i)
         for (uint32_t j = 0; j < n; ++j) {
             const float x = T_host[(size_t)i * n + j];
-            if (i != j && !(x > 0.0f && std::isfinite(x))) return RR_ERR_ARG;
+            if ((i != j || flags) && !(x > 0.0f && std::isfinite(x))) return RR_ERR_ARG;
         }
     DeviceFacts f;
     int32_t rc = device_facts(&f);
@@ -300,7 +304,7 @@ extern "C" int32_t rr_cluster(const float *T_host, uint32_t n, void *scratch_dev
     uint8_t *work = (uint8_t *)scratch_dev + sizeof(ScratchHeader);
     RR_CUDA(cudaMemcpyAsync(work + lay.off_T, T_host, sizeof(float) * n * n, cudaMemcpyHostToDevice,
                             stream));
-    cluster_kernel<<<1, kClusterThreads, 0, stream>>>(work, n);
+    cluster_kernel<<<1, kClusterThreads, 0, stream>>>(work, n, flags);
     RR_CUDA(cudaGetLastError());
     ClusterOut out;
     RR_CUDA(cudaMemcpyAsync(&out, work + lay.off_out, sizeof(out), cudaMemcpyDeviceToHost, stream));

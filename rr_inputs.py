@@ -53,11 +53,12 @@ def usable_region_bytes(free_bytes: int, frac: float = 0.95) -> int:
 
 def planted_matrix(group_sizes, drop: float, seed: int, tpc_drop: float = 0.10,
                    background: float = 0.02, sigma: float = 0.02, shuffle: bool = True,
-                   base_gbps: float = 100.0):
+                   base_gbps: float = 100.0, solo_spread: float = 0.0):
     """A synthetic SM x SM pair-throughput matrix with a planted partition.
 
-    SMs come in TPC pairs (ids 2k, 2k+1).  Entry (i, j):
-      base * (1 - drop [same group]) * (1 - tpc_drop [same TPC])
+    SMs come in TPC pairs (ids 2k, 2k+1).  SM i alone runs at solo_i = base/2 * (1 + solo_spread
+    * U(-1,1)) (the diagonal).  Entry (i, j):
+      (solo_i + solo_j) * (1 - drop [same group]) * (1 - tpc_drop [same TPC])
            * (1 - background [the two SMs lie in different halves of the chip])
            * (1 + sigma * N(0,1)),   drawn independently for (i,j) and (j,i).
     Group sizes must be even.  With ``shuffle`` the TPCs are permuted at random so groups are
@@ -81,12 +82,15 @@ def planted_matrix(group_sizes, drop: float, seed: int, tpc_drop: float = 0.10,
     same_g = grp[:, None] == grp[None, :]
     same_t = tpc[:, None] == tpc[None, :]
     diff_h = half[:, None] != half[None, :]
-    T = np.full((n, n), base_gbps, dtype=np.float64)
+    solo = 0.5 * base_gbps * (1.0 + solo_spread * rng.uniform(-1.0, 1.0, n))
+    if solo_spread == 0.0:
+        solo = np.full(n, 0.5 * base_gbps)
+    T = solo[:, None] + solo[None, :]
     T *= np.where(same_g, 1.0 - drop, 1.0)
     T *= np.where(same_t, 1.0 - tpc_drop, 1.0)
     T *= np.where(diff_h, 1.0 - background, 1.0)
     T *= 1.0 + sigma * rng.standard_normal((n, n))
-    np.fill_diagonal(T, base_gbps * 0.55)  # solo runs: one SM alone
+    T[np.arange(n), np.arange(n)] = solo * (1.0 + 0.25 * sigma * rng.standard_normal(n))
     # canonical truth labels
     truth = np.empty(n, dtype=np.int32)
     seen = {}

@@ -97,12 +97,16 @@ def test_other_entry_points_reject_bad_arguments():
     T[2, 3] = np.nan
     g = np.zeros(8, np.int32)
     ng = ctypes.c_uint32()
-    assert lib.rr_cluster(T.ctypes.data, 8, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    assert lib.rr_cluster(T.ctypes.data, 8, 0, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
     T[2, 3] = -1
-    assert lib.rr_cluster(T.ctypes.data, 8, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    assert lib.rr_cluster(T.ctypes.data, 8, 0, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
     T[2, 3] = 1
-    assert lib.rr_cluster(T.ctypes.data, 1, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
-    assert lib.rr_cluster(T.ctypes.data, 8, FAKE + 4, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ALIGN
+    assert lib.rr_cluster(T.ctypes.data, 8, 2, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    T[4, 4] = 0   # solo normalisation needs a valid diagonal
+    assert lib.rr_cluster(T.ctypes.data, 8, 1, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    T[4, 4] = 1
+    assert lib.rr_cluster(T.ctypes.data, 1, 0, FAKE, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ARG
+    assert lib.rr_cluster(T.ctypes.data, 8, 0, FAKE + 4, g.ctypes.data, ctypes.byref(ng), None, None, 0) == rr.RR_ERR_ALIGN
 
 
 def test_make_windows_matches_oracle():

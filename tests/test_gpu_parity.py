@@ -231,6 +231,11 @@ def test_cluster_matches_oracle(dev, sizes, drop):
         assert G == oG and np.array_equal(g, og)
         assert np.array_equal(h, oh)                       # same divisions, same doubles
         assert conf == oconf or (np.isinf(conf) and np.isinf(oconf))
+        T2, _ = rr_inputs.planted_matrix(sizes, drop, seed=seed, solo_spread=0.15)
+        g, G, conf, h = rr.rr_cluster(T2, dev.scratch, flags=rr.RR_CLUSTER_SOLO_NORMALISE)
+        og, oG, oconf, oh = oracle.cluster(T2, solo_normalise=True)
+        assert G == oG and np.array_equal(g, og) and np.array_equal(h, oh)
+        assert conf == oconf or (np.isinf(conf) and np.isinf(oconf))
         if drop >= 0.06 and len(sizes) >= 6 and sum(sizes) // 3 >= len(sizes):
             assert G == len(sizes) and np.array_equal(g, truth)
 

@@ -116,3 +116,30 @@ def test_ties_break_towards_smallest_pair():
     T = np.full((9, 9), 50.0, np.float32)
     g, G, conf, heights = oracle.cluster(T)
     assert G == 1 and conf == 0.0 and np.all(heights == 1048576.0)
+
+
+def test_solo_normalisation_removes_per_sm_speed_differences():
+    # SMs whose solo rates differ by +-15 % blur a 10 % contention drop in the raw matrix; dividing
+    # each pair by its two solo rates (the diagonal) restores exact recovery
+    raw_ok = norm_ok = 0
+    for s in range(40):
+        sizes = rr_inputs.random_group_sizes(3000 + s)
+        T, truth = rr_inputs.planted_matrix(sizes, 0.10, seed=s, solo_spread=0.15)
+        g, G, _, _ = oracle.cluster(T)
+        raw_ok += G == len(sizes) and np.array_equal(g, truth)
+        g, G, conf, _ = oracle.cluster(T, solo_normalise=True)
+        norm_ok += G == len(sizes) and np.array_equal(g, truth)
+    assert norm_ok == 40 and raw_ok < 40
+
+
+def test_solo_normalisation_is_scale_free_and_checks_the_diagonal():
+    T, truth = rr_inputs.planted_matrix([6, 8, 6, 8, 6], 0.3, seed=2, solo_spread=0.1)
+    g1, G1, c1, h1 = oracle.cluster(T, solo_normalise=True)
+    g2, G2, c2, h2 = oracle.cluster(T * 4.0, solo_normalise=True)   # power-of-two scale: exact
+    assert G1 == G2 == 5 and np.array_equal(g1, g2) and np.array_equal(h1, h2)
+    assert np.array_equal(g1, truth)
+    B = T.copy()
+    B[3, 3] = 0.0
+    with pytest.raises(oracle.OracleError):
+        oracle.cluster(B, solo_normalise=True)
+    oracle.cluster(B)      # without the flag the diagonal is ignored
