@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the full-memory random-line-read path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Metric (the benchmark spec): random 128-B line read GB/s over the full HBM with every SM group held
+to its own window below the measured translation reach, next to the unrestricted rate over the
+same region.  One step = one launch of the persistent read kernel over ~95 % of free HBM:
+every warp on every SM performs 2^8 x 64 random 128-byte line reads inside its group's window.
+
+Before the timed region each rank calibrates its own GPU (the layout differs card to card):
+fill, pair-probe matrix, clustering into SM groups, size sweep and reach, window assignment.
+Those calibration results and their timings are reported under "calibration".
+
+N > 1 runs N independent replicas (one process per GPU, no data-path collective): the layout
+discovery is per card and the reads touch local HBM only.  value = all ranks' bytes / slowest
+rank's time.
+
+--impl reference times the CPU oracle (the plain definition of the same path) on host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import datetime
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np  # noqa: E402
+
+GiB = 1 << 30
+READS_PER_ITER = 1 << 8       # configs[1] / [4]: 2^8 reads per warp per iteration
+ITERS_PER_STEP = 64           # one launch runs 64 iterations of the same stream
+WARPS_PER_SM = 32
+SEED = 23                     # configs[4]
+METRIC = "random 128-B line read GB/s over full HBM (grouped windows)"
+NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm: no GPU to ask
+
+
+def _peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        return json.loads(p.read_text()), "measured"
+    return {"hbm_gbs": 6650.0}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(device_index)],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def wait_first_sample(self, timeout=5.0):
+        t0 = time.time()
+        while self.proc and time.time() - t0 < timeout:
+            if os.path.getsize(self.file.name) > 0:
+                return
+            time.sleep(0.05)
+
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        if self.proc:
+            self.proc.terminate()        # the exact PID we started
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.file.flush()
+        rows = Path(self.file.name).read_text().splitlines()
+        os.unlink(self.file.name)
+        inside, everything = [], []
+        for r in rows:
+            c = [x.strip() for x in r.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rec = (float(c[1]), float(c[2]), c[4:9])
+            except ValueError:
+                continue
+            everything.append(rec)
+            if t_begin - 0.05 <= ts <= t_end + 0.05:
+                inside.append(rec)
+        use = inside if len(inside) >= 2 else everything
+        if not use:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"], "samples": 0}
+        names = ["active", "hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                 "sw_power_cap"]
+        reasons = set()
+        for _, _, flags in use:
+            for name, f in zip(names[1:], flags[1:]):
+                if f.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(r[0] for r in use), "sm_max_mhz": use[0][1],
+                "reasons": sorted(reasons), "samples": len(use),
+                "during_timed_region": len(inside) >= 2}
+
+
+def _oracle_sample(region_bytes, nsm, groups, windows, target_seconds):
+    """Times the oracle, as it stands, on all warps of the workload for a bounded number of reads
+    per warp.  Returns (GB/s-equivalent, reads_per_warp, seconds, checksums)."""
+    import oracle
+    wps = WARPS_PER_SM
+    t0 = time.time()
+    oracle.read_per_sm(region_bytes, 1, nsm, wps, 8, SEED, group_of_sm=groups, windows=windows)
+    per_read = max((time.time() - t0) / 8, 1e-6)
+    reads = int(max(8, min(1 << 20, target_seconds / per_read)))
+    t0 = time.time()
+    out = oracle.read_per_sm(region_bytes, 1, nsm, wps, reads, SEED, group_of_sm=groups,
+                             windows=windows)
+    dt = time.time() - t0
+    active = int((np.asarray(groups) != 0xFFFF).sum()) if groups is not None else nsm
+    return active * wps * reads * 128 / dt * 1e-9, reads, dt, out
+
+
+def run_reference(args):
+    """The oracle on host cores, on the same metric and workload shape (bounded sample per step)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    import rr_inputs
+    oracle.build()
+    nsm, n_groups = 148, 24
+    groups = rr_inputs.synthetic_group_map(nsm, n_groups, seed=1)
+    windows, _ = oracle.make_windows(NOMINAL_REGION, 1, 32 * GiB, n_groups)
+    per_step = max(0.5, min(4.0, 60.0 / max(args.steps + args.warmup, 1)))
+    gbps, reads, _, _ = _oracle_sample(NOMINAL_REGION, nsm, groups, windows, per_step)
+    for _ in range(args.warmup):
+        oracle.read_per_sm(NOMINAL_REGION, 1, nsm, WARPS_PER_SM, reads, SEED, group_of_sm=groups,
+                           windows=windows)
+    t0 = time.time()
+    for k in range(args.steps):
+        oracle.read_per_sm(NOMINAL_REGION, 1, nsm, WARPS_PER_SM, reads, SEED, group_of_sm=groups,
+                           windows=windows, first_read=k * reads)
+    dt = time.time() - t0
+    value = args.steps * nsm * WARPS_PER_SM * reads * 128 / dt * 1e-9
+    cores = oracle.n_threads()
+    sample = (f"all {nsm * WARPS_PER_SM} warps x {reads} reads per step "
+              f"(a full step is {READS_PER_ITER * ITERS_PER_STEP} reads per warp)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": {"workload": "cfg4 grouped full-memory random 128-B reads (CPU oracle, "
+                               "regenerating buffer contents)", "region_bytes": NOMINAL_REGION,
+                   "n_groups": n_groups, "window_bytes": 32 * GiB, "seed": SEED},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+    }))
+    return 0
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2405_11425_b200 import binding as rr
+    from paper_2405_11425_b200 import build as rr_build
+    from paper_2405_11425_b200.pipeline import Session, aggregate_throughput
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; this path has no CPU fallback "
+                         "(use --impl reference for the oracle timing)")
+    if rank == 0:
+        rr_build.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    peaks, peak_kind = _peaks()
+
+    # ---- calibration (untimed): fill, groups, reach, windows --------------------------------
+    ses = Session()
+    fill_gbps = ses.fill()
+    fill_gbps = max(fill_gbps, ses.fill())
+    groups = ses.discover_groups(total_reads=args.probe_reads, repeats=args.probe_repeats)
+    reach = ses.measure_reach()
+    N = ses.region_bytes
+    unrestricted_full, _ = ses.read(N, seed=SEED, reads_per_warp=READS_PER_ITER * 16)
+    if reach.cliff:
+        sweep_sizes = {"reach/4": reach.reach_bytes // 4, "reach/2": reach.reach_bytes // 2,
+                       "reach": reach.reach_bytes, "2*reach": 2 * reach.reach_bytes, "N/2": N // 2}
+        headline = "reach/2"
+    else:
+        sweep_sizes = {"N/8": N // 8, "N/4": N // 4, "N/2": N // 2, "N": N}
+        headline = "N/4"
+    window_sweep = {}
+    for name, S in sweep_sizes.items():
+        win, cov = ses.windows(groups, S)
+        g, _ = ses.read(N, seed=SEED, reads_per_warp=READS_PER_ITER * 16,
+                        group_of_sm=groups.group_of_sm, windows=win)
+        window_sweep[name] = {"window_gib": S / GiB, "coverage": cov, "gbps": g}
+    S = sweep_sizes[headline]
+    windows, coverage = ses.windows(groups, S)
+    in_window, _ = ses.read(min(S, N), seed=SEED, reads_per_warp=READS_PER_ITER * 16)
+    ctrl_groups, ctrl_win, _ = ses.naive_control(S, SEED)
+    naive_control, _ = ses.read(N, seed=SEED, reads_per_warp=READS_PER_ITER * 16,
+                                group_of_sm=ctrl_groups, windows=ctrl_win)
+
+    # ---- timed region: device-resident, asynchronous launches -------------------------------
+    reads = READS_PER_ITER * ITERS_PER_STEP
+    stream = torch.cuda.current_stream()
+
+    def params(step):
+        return ses.params(N, W=1, warps_per_sm=WARPS_PER_SM, reads_per_warp=reads,
+                          first_read=step * reads, seed=SEED, group_of_sm=groups.group_of_sm,
+                          windows=windows)
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.wait_first_sample()
+    for k in range(args.warmup):
+        rr.rr_random_read(params(k), ses.out, ses.scratch, timed=False)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.time()
+    e0.record(stream)
+    for k in range(args.steps):
+        rr.rr_random_read(params(args.warmup + k), ses.out, ses.scratch, timed=False)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t_end = time.time()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    seconds = e0.elapsed_time(e1) * 1e-3
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
+    last = rr.rr_read_report(params(args.warmup + args.steps - 1), ses.scratch)
+    step_bytes = ses.nsm * WARPS_PER_SM * reads * 128
+    assert last.bytes == step_bytes and last.sms_covered == ses.nsm
+    tot_bytes, max_seconds = aggregate_throughput(step_bytes * args.steps, seconds)
+    value = tot_bytes / max_seconds * 1e-9
+
+    # ---- end to end: synchronous call, tables in, checksums and timing record out -----------
+    host_out = torch.empty((ses.nsm * WARPS_PER_SM, 2), dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k in range(e2e_steps):
+        rr.rr_random_read(params(k), ses.out, ses.scratch, timed=True)
+        host_out.copy_(ses.out[: ses.nsm * WARPS_PER_SM], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_seconds = time.perf_counter() - t0
+    e2e_bytes, e2e_max = aggregate_throughput(step_bytes * e2e_steps, e2e_seconds)
+    h2d = ses.nsm * 2 + groups.n_groups * 8 + 128          # tables + scalars in the launch
+    d2h = host_out.numel() * 4 + 8208                      # checksums + timing records
+
+    # ---- oracle beside it: parity on every warp of a bounded sample, and its timing ---------
+    cpu = None
+    parity = None
+    if rank == 0:
+        import oracle
+        oracle.build()
+        o_gbps, o_reads, o_dt, o_out = _oracle_sample(N, ses.nsm, groups.group_of_sm, windows, 12.0)
+        p = ses.params(N, W=1, warps_per_sm=WARPS_PER_SM, reads_per_warp=o_reads, seed=SEED,
+                       group_of_sm=groups.group_of_sm, windows=windows)
+        rr.rr_random_read(p, ses.out, ses.scratch)
+        same = np.array_equal(ses.checksums(ses.nsm * WARPS_PER_SM), o_out)
+        parity = {"warps": ses.nsm * WARPS_PER_SM, "reads_per_warp": o_reads, "bit_exact": bool(same)}
+        cpu = {"value": o_gbps, "unit": "GB/s", "cores": oracle.n_threads(), "kind": "oracle",
+               "sample": f"all {ses.nsm * WARPS_PER_SM} warps x {o_reads} reads of the same "
+                         f"grouped workload ({o_dt:.1f} s)"}
+
+    if rank == 0:
+        peak = float(peaks["hbm_gbs"])
+        achieved = step_bytes / (seconds / args.steps) * 1e-9
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": max_seconds / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {
+                "workload": "cfg4 grouped full-memory random 128-B line reads: every SM group "
+                            "held to its own window (" + headline + "), all warps, seed 23",
+                "region_bytes": N, "region_gib": N / GiB, "line_bytes": 128,
+                "warps_per_sm": WARPS_PER_SM, "reads_per_warp_per_step": reads,
+                "window_bytes": S, "coverage": coverage, "n_groups": groups.n_groups,
+                "l2": "inputs (region) far larger than L2; no flush needed",
+                "parallelism": "replicas" if world > 1 else "single GPU",
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_bytes / e2e_max * 1e-9, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind} (copy, read+write)",
+                         "traffic": TRAFFIC_PER_ALGORITHMIC_BYTE * step_bytes
+                         if TRAFFIC_PER_ALGORITHMIC_BYTE else None,
+                         "theoretical_gbps": ses.info["theoretical_gbps"],
+                         "frac_of_theoretical": achieved / ses.info["theoretical_gbps"]},
+            "cpu_baseline": cpu,
+            "parity": parity,
+            "calibration": {
+                "device": ses.info["name"], "uuid": ses.info["uuid"], "nsm": ses.nsm,
+                "fill_gbps": fill_gbps,
+                "probe": {"seconds": groups.probe_seconds, "pairs": ses.nsm * (ses.nsm + 1) // 2,
+                          "reads_per_pair": args.probe_reads, "repeats": args.probe_repeats,
+                          "overlap_min": groups.overlap_min},
+                "groups": {"n": groups.n_groups, "confidence": groups.confidence,
+                           "sizes": groups.sizes, "group_of_sm": groups.group_of_sm.tolist()},
+                "reach": {"cliff": reach.cliff, "plateau_gbps": reach.plateau_gbps,
+                          "reach_gib": reach.reach_bytes / GiB,
+                          "sweep": [[s / GiB, g] for s, g in reach.sweep]},
+                "unrestricted_full_gbps": unrestricted_full,
+                "unrestricted_in_window_gbps": in_window,
+                "naive_per_sm_control_gbps": naive_control,
+                "window_sweep": window_sweep,
+            },
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+# DRAM bytes moved per algorithmic byte by the read kernel, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over lines x 128 B); None = not captured.
+TRAFFIC_PER_ALGORITHMIC_BYTE = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--probe-reads", type=int, default=1 << 18)
+    ap.add_argument("--probe-repeats", type=int, default=3)
+    args = ap.parse_args()
+    if args.steps < 1:
+        ap.error("--steps must be >= 1")
+    return run_reference(args) if args.impl == "reference" else run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
