@@ -49,6 +49,7 @@ extern "C" {
 #define RR_ERR_CHECK (-8)        /* checked variant saw an address outside its window; the      */
                                  /* offending loads were skipped                                */
 #define RR_ERR_UNSUPPORTED (-9)  /* device is not the one this library was built for            */
+#define RR_ERR_STATIC_LIMIT (-10) /* rr_random_read_static: request exceeds its built-in scratch */
 
 /* ---- limits ---- */
 #define RR_MAX_SM 256u      /* SM ids the tables can hold (B200 has 148)                       */
@@ -163,6 +164,33 @@ int32_t rr_random_read(const rr_read_params_t *params /*HOST*/, void *out_dev /*
  * RR_ERR_SM_UNCOVERED / RR_ERR_CHECK like the timed form of rr_random_read.                   */
 int32_t rr_read_report(const rr_read_params_t *params /*HOST*/, const void *scratch_dev,
                        rr_result_t *res /*HOST*/, void *stream);
+
+/* ---- random line reads for callers that cannot allocate device memory ----------------------
+ * (The paper has no counterpart: this is a packaging variant of rr_random_read.)
+ *
+ * Some callers have no way to hand the library a scratch buffer: code running inside another
+ * framework's memory pool that may not call cudaMalloc, a plugin loaded after the host
+ * application has claimed all device memory, or a hook that runs where allocation is forbidden.
+ * For them this entry point performs exactly the read rr_random_read performs, but keeps the
+ * claim table, status words and per-block timing records in a fixed array that is part of the
+ * library image (RR_STATIC_SCRATCH_BYTES bytes, resident on every GPU that loads the library,
+ * until the process exits).  It calls no allocation routine of any kind, and creates no events:
+ * res->seconds_event is 0 and res->gbps is computed from the device-side timers.
+ *
+ * Limits: at most RR_STATIC_MAX_SM SMs and one block per SM (warps_per_sm <= 32); anything
+ * larger returns RR_ERR_STATIC_LIMIT before launching.  All other arguments, outputs and
+ * status codes are those of rr_random_read (the caller still passes buf and out_dev).
+ *
+ * The first call on each device looks up the device address of the built-in array (the device
+ * must be current); make that first call outside any stream capture.  Every call on a device
+ * shares the one array, which still holds the previous call's contents, and clears it before
+ * launching; two calls that overlap on the GPU (for instance on different streams) therefore
+ * race on it: keep calls on one device in stream order.  res == NULL queues the work and
+ * returns without waiting.                                                                    */
+#define RR_STATIC_MAX_SM 192u
+#define RR_STATIC_SCRATCH_BYTES 5888u
+int32_t rr_random_read_static(const rr_read_params_t *params /*HOST*/, void *out_dev /*DEVICE*/,
+                              rr_result_t *res /*HOST or NULL*/, void *stream);
 
 /* ---- A6: two-SM contention probe -----------------------------------------------------------
  * Paper, Section 2.2: "if we run our memory access kernel with only two SMs, we expect ... a

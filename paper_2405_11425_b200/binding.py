@@ -18,6 +18,8 @@ LIB_PATH = _PKG / "librr.so"
 RR_OK = 0
 RR_ERR_ARG, RR_ERR_ALIGN, RR_ERR_RANGE, RR_ERR_MAP, RR_ERR_CUDA = -1, -2, -3, -4, -5
 RR_ERR_SM_UNCOVERED, RR_ERR_TIMEOUT, RR_ERR_CHECK, RR_ERR_UNSUPPORTED = -6, -7, -8, -9
+RR_ERR_STATIC_LIMIT = -10
+RR_STATIC_MAX_SM, RR_STATIC_SCRATCH_BYTES = 192, 5888
 RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 64, 0xFFFF
 RR_MODE_LOGICAL, RR_MODE_PER_SM = 0, 1
 RR_INDEX_RANDOM, RR_INDEX_STRIDE = 0, 1
@@ -26,7 +28,7 @@ RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED = 0, 1
 EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
     "rr_random_read", "rr_read_report", "rr_probe_pair", "rr_probe_matrix_scratch_bytes",
-    "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach",
+    "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach", "rr_random_read_static",
 )
 
 
@@ -119,6 +121,8 @@ def _load():
     lib.rr_fill.argtypes = [p, u64, p]
     lib.rr_random_read.restype = i32
     lib.rr_random_read.argtypes = [p, p, p, p, p]
+    lib.rr_random_read_static.restype = i32
+    lib.rr_random_read_static.argtypes = [p, p, p, p]
     lib.rr_read_report.restype = i32
     lib.rr_read_report.argtypes = [p, p, p, p]
     lib.rr_probe_pair.restype = i32
@@ -221,6 +225,18 @@ def rr_random_read(params: ReadParams, out, scratch, *, timed: bool = True, stre
                                 ctypes.byref(res) if timed else None, _stream(stream))
     _check(rc, "rr_random_read")
     return _result(res) if timed else None
+
+
+def rr_random_read_static(params: ReadParams, out, *, report: bool = True, stream=None):
+    """rr_random_read for callers that cannot allocate: the scratch is built into the library.
+
+    `report` = wait and return a ReadResult (device-side timing only), else queue and return
+    None.  Calls on one device share the built-in scratch and must not overlap."""
+    res = _Result()
+    rc = _load().rr_random_read_static(ctypes.byref(params.c), _dev(out),
+                                       ctypes.byref(res) if report else None, _stream(stream))
+    _check(rc, "rr_random_read_static")
+    return _result(res) if report else None
 
 
 def rr_read_report(params: ReadParams, scratch, stream=None) -> ReadResult:

@@ -56,6 +56,9 @@ extern "C" const char *rr_strerror(int32_t code)
         case RR_ERR_TIMEOUT: return "device-side wait ran out";
         case RR_ERR_CHECK: return "checked variant rejected an address";
         case RR_ERR_UNSUPPORTED: return "unsupported device";
+        case RR_ERR_STATIC_LIMIT:
+            return "request exceeds the built-in scratch of rr_random_read_static "
+                   "(at most 192 SMs, at most 32 warps per SM)";
         default: return "unknown status";
     }
 }

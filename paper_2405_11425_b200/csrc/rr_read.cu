@@ -699,3 +699,106 @@ extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint6
     if (overlap_min_host) *overlap_min_host = overlap_min;
     return RR_OK;
 }
+
+// ---- rr_random_read_static: the same read with built-in scratch ---------------------------------
+// For callers that cannot obtain device memory of their own (see rr.h).  The scratch lives in a
+// file-scope device array; in host code its name is only a handle, so the device address is
+// fetched once per device with cudaGetSymbolAddress and cached here.
+#include <mutex>
+
+namespace rr {
+
+constexpr uint32_t kStaticMaxSm = RR_STATIC_MAX_SM;
+// header words + claim table + one timing record per SM (one block per SM only)
+constexpr size_t kStaticUsedBytes = offsetof(ScratchHeader, rec) + sizeof(BlockRecord) * kStaticMaxSm;
+static_assert(kStaticUsedBytes <= RR_STATIC_SCRATCH_BYTES, "static scratch too small for its limits");
+static_assert(kStaticMaxSm <= RR_MAX_SM, "static limit exceeds the table size");
+
+static __device__ __align__(256) unsigned char g_static_scratch[RR_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void *g_static_ptr[kMaxDevices];  // device address of g_static_scratch, per device ordinal
+
+// Device address of the built-in scratch on the current device (first call per device asks the
+// runtime; later calls read the cache).
+static int32_t static_scratch_address(int device, void **out)
+{
+    if (device < 0 || device >= kMaxDevices) return RR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void *p = nullptr;
+        RR_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p || (uintptr_t)p % 256u) return RR_ERR_ALIGN;
+        g_static_ptr[device] = p;
+    }
+    *out = g_static_ptr[device];
+    return RR_OK;
+}
+
+}  // namespace rr
+
+extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_dev, rr_result_t *res,
+                                         void *stream_)
+{
+    uint32_t U = 0;
+    // validate against a stand-in scratch address first: argument errors come before any CUDA call
+    int32_t rc = validate_read(p, out_dev, (const void *)256, &U);
+    if (rc != RR_OK) return rc;
+    if (p->mode == RR_MODE_PER_SM && (p->warps_per_sm > 32 || p->nsm > kStaticMaxSm))
+        return RR_ERR_STATIC_LIMIT;
+    DeviceFacts f;
+    rc = device_facts(&f);
+    if (rc != RR_OK) return rc;
+    if ((uint32_t)f.nsm > kStaticMaxSm) return RR_ERR_STATIC_LIMIT;
+    Geometry g;
+    rc = geometry(p, f, &g);
+    if (rc != RR_OK) return rc;
+    if (g.cps != 1 || g.grid > kStaticMaxSm) return RR_ERR_STATIC_LIMIT;
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant == RR_VARIANT_LDG_CHECKED);
+    if (!kernel) return RR_ERR_ARG;
+    void *scratch = nullptr;
+    rc = static_scratch_address(f.device, &scratch);
+    if (rc != RR_OK) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    size_t smem = 0;
+    if (p->mode == RR_MODE_PER_SM) {
+        rc = ballast_for_occupancy(kernel, (int)g.block, 1, f, &smem);
+        if (rc != RR_OK) return rc;
+    }
+    ReadArgs a;
+    a.buf = (const char *)p->buf;
+    a.region_bytes = p->region_bytes;
+    a.reads = p->reads_per_warp;
+    a.first_read = p->first_read;
+    a.key_seed = sm64(p->seed);
+    a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
+    a.mode = p->mode;
+    a.index_mode = p->index_mode;
+    a.n_warps = p->n_warps;
+    a.wps = g.wps;
+    a.wpc = g.wpc;
+    a.cps = g.cps;
+    a.nsm = (uint32_t)f.nsm;
+    a.n_groups = p->group_of_sm ? p->n_groups : 0;
+    a.out = (uint2 *)out_dev;
+    a.scratch = (ScratchHeader *)scratch;
+    Tables tab;
+    std::memset(&tab, 0, sizeof(tab));
+    if (p->group_of_sm) {
+        std::memcpy(tab.group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
+        std::memcpy(tab.windows, p->windows, sizeof(rr_window_t) * p->n_groups);
+    }
+    // the array keeps the previous call's claims, counters and records: clear them
+    RR_CUDA(cudaMemsetAsync(scratch, 0, kStaticUsedBytes, stream));
+    if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
+        RR_CUDA(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
+    kernel<<<g.grid, g.block, smem, stream>>>(a, tab);
+    RR_CUDA(cudaGetLastError());
+    if (!res) return RR_OK;
+    static thread_local ScratchHeader h;
+    std::memset(&h, 0, sizeof(h));
+    RR_CUDA(cudaMemcpyAsync(&h, scratch, kStaticUsedBytes, cudaMemcpyDeviceToHost, stream));
+    RR_CUDA(cudaStreamSynchronize(stream));
+    return decode(p, g, f, h, 0.0, res);
+}
