@@ -54,7 +54,7 @@ extern "C" {
 /* ---- limits ---- */
 #define RR_MAX_SM 256u      /* SM ids the tables can hold (B200 has 148)                       */
 #define RR_MAX_GROUPS 256u  /* one window per group; the naive control uses one group per SM   */
-#define RR_MAX_WARPS_PER_SM 64u
+#define RR_MAX_WARPS_PER_SM 32u /* one 1024-thread block per SM                                 */
 #define RR_SM_INACTIVE 0xFFFFu
 
 /* ---- enums (plain integers in the structs) ---- */
@@ -131,7 +131,7 @@ typedef struct {
     uint32_t mode;              /* RR_MODE_*                                                   */
     uint32_t index_mode;        /* RR_INDEX_*                                                  */
     uint32_t n_warps;           /* LOGICAL                                                     */
-    uint32_t warps_per_sm;      /* PER_SM: 1..32, or 34..64 even (two blocks per SM)           */
+    uint32_t warps_per_sm;      /* PER_SM: 1..RR_MAX_WARPS_PER_SM (one block per SM)           */
     uint32_t nsm;               /* PER_SM: SM count of the device, 0 = query                   */
     uint64_t reads_per_warp;
     uint64_t first_read;
@@ -177,8 +177,8 @@ int32_t rr_read_report(const rr_read_params_t *params /*HOST*/, const void *scra
  * until the process exits).  It calls no allocation routine of any kind, and creates no events:
  * res->seconds_event is 0 and res->gbps is computed from the device-side timers.
  *
- * Limits: at most RR_STATIC_MAX_SM SMs and one block per SM (warps_per_sm <= 32); anything
- * larger returns RR_ERR_STATIC_LIMIT before launching.  All other arguments, outputs and
+ * Limit: at most RR_STATIC_MAX_SM SMs (the device's count, or the nsm passed in); a larger
+ * count returns RR_ERR_STATIC_LIMIT before launching.  All other arguments, outputs and
  * status codes are those of rr_random_read (the caller still passes buf and out_dev).
  *
  * The first call on each device looks up the device address of the built-in array (the device
@@ -237,6 +237,18 @@ int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint6
 int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratch_dev /*DEVICE*/,
                    int32_t *group_of_sm_host, uint32_t *n_groups, double *confidence,
                    double *heights_host, void *stream);
+
+/* ---- cross-check of the layout by cluster placement -----------------------------------------
+ * Paper, Section 1.1: "there is no simple way to determine which GPC each SM is on".  Blocks of
+ * one thread-block cluster always run on one GPC, so this call launches clusters of 2..8 small
+ * blocks, records %smid per block and merges SMs that shared a cluster: gpc_of_sm_host[nsm]
+ * (HOST) receives a GPC label per SM (numbered by smallest SM id), *n_gpcs their count.  No
+ * timing is involved; every contention group found by rr_cluster on a probe matrix should lie
+ * inside one of these GPCs (Section 2.2 found groups finer than GPCs).  nsm = the device's SM
+ * count.  Synchronous; uses rr_scratch_bytes() of scratch.  RR_ERR_SM_UNCOVERED if some SM never
+ * received a block.                                                                            */
+int32_t rr_gpc_map(void *scratch_dev /*DEVICE*/, int32_t *gpc_of_sm_host /*HOST*/,
+                   uint32_t *n_gpcs, uint32_t nsm, void *stream);
 
 /* ---- A9 policy: windows per group (host only) ----------------------------------------------
  * Paper, Section 1.3 ("restricted to a 64GB window (or, say, half the memory for simplicity)")

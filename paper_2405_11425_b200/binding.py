@@ -20,7 +20,7 @@ RR_ERR_ARG, RR_ERR_ALIGN, RR_ERR_RANGE, RR_ERR_MAP, RR_ERR_CUDA = -1, -2, -3, -4
 RR_ERR_SM_UNCOVERED, RR_ERR_TIMEOUT, RR_ERR_CHECK, RR_ERR_UNSUPPORTED = -6, -7, -8, -9
 RR_ERR_STATIC_LIMIT = -10
 RR_STATIC_MAX_SM, RR_STATIC_SCRATCH_BYTES = 192, 5888
-RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 64, 0xFFFF
+RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0xFFFF
 RR_MODE_LOGICAL, RR_MODE_PER_SM = 0, 1
 RR_INDEX_RANDOM, RR_INDEX_STRIDE = 0, 1
 RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED = 0, 1
@@ -29,6 +29,7 @@ EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
     "rr_random_read", "rr_read_report", "rr_probe_pair", "rr_probe_matrix_scratch_bytes",
     "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach", "rr_random_read_static",
+    "rr_gpc_map",
 )
 
 
@@ -133,6 +134,8 @@ def _load():
     lib.rr_probe_matrix.argtypes = [p, u64, u64, u32, u64, u32, p, u32, p, p, p, p]
     lib.rr_cluster.restype = i32
     lib.rr_cluster.argtypes = [p, u32, u32, p, p, p, p, p, p]
+    lib.rr_gpc_map.restype = i32
+    lib.rr_gpc_map.argtypes = [p, p, p, u32, p]
     lib.rr_make_windows.restype = i32
     lib.rr_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p]
     lib.rr_reach.restype = i32
@@ -283,6 +286,15 @@ def rr_cluster(T, scratch, flags: int = 0, stream=None):
                               ctypes.byref(ng), ctypes.byref(conf), heights.ctypes.data,
                               _stream(stream)), "rr_cluster")
     return groups, int(ng.value), float(conf.value), heights[: n - 1]
+
+
+def rr_gpc_map(scratch, nsm: int, stream=None):
+    """Returns (gpc_of_sm int32[nsm], n_gpcs) from thread-block-cluster placement."""
+    g = np.zeros(nsm, dtype=np.int32)
+    ng = ctypes.c_uint32()
+    _check(_load().rr_gpc_map(_dev(scratch), g.ctypes.data, ctypes.byref(ng), nsm,
+                              _stream(stream)), "rr_gpc_map")
+    return g, int(ng.value)
 
 
 def rr_make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int, policy: int = 0,

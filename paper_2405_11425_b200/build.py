@@ -15,7 +15,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 INCLUDE = ROOT / "include"
 LIB = PKG / "librr.so"
-SOURCES = ["rr_host.cu", "rr_fill.cu", "rr_read.cu", "rr_cluster.cu"]
+SOURCES = ["rr_host.cu", "rr_fill.cu", "rr_read.cu", "rr_cluster.cu", "rr_gpc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", f"-I{INCLUDE}", f"-I{CSRC}",
@@ -62,7 +62,8 @@ def build(force: bool = False, verbose: bool = False) -> Path:
             raise RuntimeError(f"nvcc failed on {src}")
         objs.append(str(obj))
     tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    subprocess.run([nvcc, "-shared", "-o", str(tmp), *objs], check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *objs],
+                   check=True)
     os.replace(tmp, LIB)
     return LIB
 

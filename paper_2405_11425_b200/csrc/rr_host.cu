@@ -58,7 +58,7 @@ extern "C" const char *rr_strerror(int32_t code)
         case RR_ERR_UNSUPPORTED: return "unsupported device";
         case RR_ERR_STATIC_LIMIT:
             return "request exceeds the built-in scratch of rr_random_read_static "
-                   "(at most 192 SMs, at most 32 warps per SM)";
+                   "(at most 192 SMs)";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,226 @@
+"""Runs the paper's experiments on the current GPU and writes report.json / report.md.
+
+    python -m paper_2405_11425_b200.report --out DIR [--quick]
+
+Experiments (paper section -> BASELINE config):
+  size sweep, unrestricted            Section 2.1, Fig. 1            configs[1]
+  line widths at 32 GiB               Section 2.1                    configs[2]
+  pair probe + clustering             Section 2.2, Fig. 2-3          configs[3]
+  single groups, group pairs          Section 2.3, Fig. 4-5          (next row 1)
+  grouped windows over all memory     Section 2.4, Fig. 6            configs[4]
+  sequential reads of the same kernel Section 2.1 ("even better")    (next row 3)
+All numbers are event-timed GB/s (10^9 B/s), median of the repetitions; nothing is computed here
+beyond bookkeeping.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+from pathlib import Path
+
+import numpy as np
+
+from . import binding as rr
+from .pipeline import GiB, Session
+
+
+def _stats(ses, region, reps=5, **kw):
+    p = ses.params(region, **kw)
+    rr.rr_random_read(p, ses.out, ses.scratch)
+    r = sorted(rr.rr_random_read(p, ses.out, ses.scratch).gbps for _ in range(reps))
+    return {"median": r[(len(r) - 1) // 2], "min": r[0], "max": r[-1]}
+
+
+def run(out_dir: Path, quick: bool = False) -> dict:
+    import torch
+    torch.cuda.set_device(0)
+    out_dir.mkdir(parents=True, exist_ok=True)
+    t_start = time.time()
+    ses = Session()
+    N = ses.region_bytes
+    R = {"device": ses.info, "region_bytes": N, "region_gib": N / GiB,
+         "alloc_conf": __import__("os").environ.get("PYTORCH_CUDA_ALLOC_CONF", "")}
+    R["fill_gbps"] = max(ses.fill(), ses.fill())
+    reads = 256 * (16 if quick else 64)
+    reps = 3 if quick else 5
+
+    # configs[0]: correctness case, rate informational
+    out0 = torch.zeros((1 << 16, 2), dtype=torch.int32, device="cuda")
+    p0 = rr.ReadParams(ses.buf, 1 * GiB, W=1, mode=rr.RR_MODE_LOGICAL, n_warps=1 << 16,
+                       reads_per_warp=16, seed=1)
+    rr.rr_random_read(p0, out0, ses.scratch)
+    R["cfg0_gbps_informational"] = rr.rr_random_read(p0, out0, ses.scratch).gbps
+
+    # configs[1]: size sweep, two occupancies
+    sizes = [s * GiB for s in (1, 4, 16, 32, 48, 64, 96, 128, 160) if s * GiB < N] + [N]
+    sweep = []
+    for n in sizes:
+        row = {"gib": n / GiB}
+        for wps in (16, 32):
+            row[f"wps{wps}"] = _stats(ses, n, reps, seed=7, reads_per_warp=reads, warps_per_sm=wps)
+        row["best"] = max(row["wps16"]["median"], row["wps32"]["median"])
+        sweep.append(row)
+    R["cfg1_size_sweep"] = sweep
+    reach = ses.measure_reach()
+    R["reach"] = {"cliff": reach.cliff, "plateau_gbps": reach.plateau_gbps,
+                  "reach_gib": reach.reach_bytes / GiB,
+                  "points": [[s / GiB, g] for s, g in reach.sweep]}
+
+    # configs[2]: widths
+    R["cfg2_widths_32gib"] = {f"{128 * W}B": _stats(ses, 32 * GiB, reps, W=W, seed=11,
+                                                    reads_per_warp=reads) for W in (1, 2, 4)}
+    # sequential control of the same kernel
+    R["stride_full"] = {f"{128 * W}B": _stats(ses, N, reps, W=W, reads_per_warp=reads,
+                                              index_mode=rr.RR_INDEX_STRIDE) for W in (1, 2, 4)}
+
+    # configs[3]: probe inside the reach (as the config says) and over everything
+    t0 = time.time()
+    g16 = ses.discover_groups(probe_region_bytes=16 * GiB,
+                              total_reads=(1 << 18) if quick else (1 << 20),
+                              repeats=3, seed=5)
+    np.save(out_dir / "probe_matrix_16gib.npy", g16.matrix)
+    gf = ses.discover_groups(total_reads=1 << 18, repeats=3, seed=5)
+    np.save(out_dir / "probe_matrix_full.npy", gf.matrix)
+    R["cfg3_probe"] = {
+        "inside_reach_16gib": {"n_groups": g16.n_groups, "confidence": g16.confidence,
+                               "seconds": g16.probe_seconds,
+                               "pair_min_med_max": _offdiag(g16.matrix)},
+        "whole_buffer": {"n_groups": gf.n_groups, "confidence": gf.confidence,
+                         "seconds": gf.probe_seconds, "sizes": gf.sizes,
+                         "group_of_sm": gf.group_of_sm.tolist(),
+                         "pair_min_med_max": _offdiag(gf.matrix),
+                         "solo_min_med_max": _mmm(np.diag(gf.matrix))},
+        "total_seconds": time.time() - t0,
+    }
+    groups = gf
+    gpc, n_gpcs = rr.rr_gpc_map(ses.scratch, ses.nsm)
+    R["gpc_map"] = {"n_components": n_gpcs, "sizes": np.bincount(gpc).tolist(),
+                    "gpc_of_sm": gpc.tolist(),
+                    "gpcs_of_group": [sorted(set(gpc[gf.group_of_sm == k].tolist()))
+                                      for k in range(gf.n_groups)]}
+
+    # next row 1: every group alone inside the reach, and pairs of groups in distinct windows
+    S = (reach.reach_bytes // 2) if reach.cliff else N // 4
+    L_S = S // 128
+    singles = []
+    for g in range(groups.n_groups):
+        gm = np.where(groups.group_of_sm == g, 0, 0xFFFF).astype(np.uint16)
+        rate = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=gm,
+                      windows=[[0, L_S]])["median"]
+        singles.append({"group": g, "sms": int((gm == 0).sum()), "gbps": rate})
+    R["single_groups"] = singles
+    pairs = []
+    ids = list(range(groups.n_groups))
+    chosen = [(a, b) for a in ids for b in ids if a < b]
+    if quick:
+        chosen = chosen[:: max(1, len(chosen) // 12)]
+    for a, b in chosen:
+        gm = np.full(ses.nsm, 0xFFFF, np.uint16)
+        gm[groups.group_of_sm == a] = 0
+        gm[groups.group_of_sm == b] = 1
+        rate = _stats(ses, N, 1, seed=23, reads_per_warp=reads, group_of_sm=gm,
+                      windows=[[0, L_S], [2 * L_S, L_S]])["median"]
+        pairs.append({"a": a, "b": b, "gbps": rate,
+                      "ratio_to_sum_of_singles": rate / (singles[a]["gbps"] + singles[b]["gbps"])})
+    R["group_pairs_distinct_windows"] = pairs
+
+    # configs[4]: window sweep, both widths, and the naive control
+    if reach.cliff:
+        wsizes = {"reach/4": reach.reach_bytes // 4, "reach/2": reach.reach_bytes // 2,
+                  "reach": reach.reach_bytes, "2*reach": 2 * reach.reach_bytes, "N/2": N // 2}
+    else:
+        wsizes = {"N/8": N // 8, "N/4": N // 4, "N/2": N // 2, "N": N}
+    cfg4 = {}
+    for W in (1, 2):
+        rows = {}
+        for name, S_w in wsizes.items():
+            win, cov = ses.windows(groups, S_w, W=W)
+            rows[name] = {"window_gib": S_w / GiB, "coverage": cov,
+                          "grouped": _stats(ses, N, reps, W=W, seed=23, reads_per_warp=reads,
+                                            group_of_sm=groups.group_of_sm, windows=win),
+                          "unrestricted_inside_one_window": _stats(
+                              ses, min(S_w, N), reps, W=W, seed=23, reads_per_warp=reads)}
+            cg, cw, ccov = ses.naive_control(S_w, 23, W=W)
+            rows[name]["naive_per_sm_control"] = _stats(ses, N, reps, W=W, seed=23,
+                                                        reads_per_warp=reads, group_of_sm=cg,
+                                                        windows=cw)
+        cfg4[f"{128 * W}B"] = {"unrestricted_full": _stats(ses, N, reps, W=W, seed=23,
+                                                           reads_per_warp=reads),
+                               "windows": rows}
+    R["cfg4_grouped"] = cfg4
+    R["seconds"] = time.time() - t_start
+    (out_dir / "report.json").write_text(json.dumps(R, indent=1))
+    (out_dir / "report.md").write_text(markdown(R))
+    return R
+
+
+def _mmm(a):
+    a = np.asarray(a, dtype=np.float64)
+    return [float(a.min()), float(np.median(a)), float(a.max())]
+
+
+def _offdiag(T):
+    n = T.shape[0]
+    return _mmm(T[~np.eye(n, dtype=bool)])
+
+
+def markdown(R: dict) -> str:
+    peak = R["device"]["theoretical_gbps"]
+    L = [f"# Random line reads on {R['device']['name']} ({R['device']['nsm_prop']} SMs, "
+         f"region {R['region_gib']:.1f} GiB, theoretical {peak:.0f} GB/s)", "",
+         f"fill: {R['fill_gbps']:.0f} GB/s", "",
+         "## Unrestricted size sweep (random 128-B lines, GB/s median [min-max])", "",
+         "| GiB | 16 warps/SM | 32 warps/SM |", "|---|---|---|"]
+    f = lambda s: f"{s['median']:.0f} [{s['min']:.0f}-{s['max']:.0f}]"  # noqa: E731
+    for r in R["cfg1_size_sweep"]:
+        L.append(f"| {r['gib']:.1f} | {f(r['wps16'])} | {f(r['wps32'])} |")
+    rc = R["reach"]
+    L += ["", f"plateau {rc['plateau_gbps']:.0f} GB/s, cliff {rc['cliff']}, reach "
+              f"{rc['reach_gib']:.0f} GiB", "", "## Line widths at 32 GiB / sequential over everything",
+          "", "| line | random 32 GiB | sequential whole buffer |", "|---|---|---|"]
+    for k in ("128B", "256B", "512B"):
+        L.append(f"| {k} | {f(R['cfg2_widths_32gib'][k])} | {f(R['stride_full'][k])} |")
+    p = R["cfg3_probe"]
+    L += ["", "## Pair probe and clustering", "",
+          f"inside the reach (16 GiB): {p['inside_reach_16gib']['n_groups']} group(s), pair GB/s "
+          f"min/med/max {p['inside_reach_16gib']['pair_min_med_max']}",
+          f"whole buffer: {p['whole_buffer']['n_groups']} groups, confidence "
+          f"{p['whole_buffer']['confidence']:.1f}, sizes {p['whole_buffer']['sizes']}, "
+          f"{p['whole_buffer']['seconds']:.1f} s",
+          f"cluster-placement components (GPCs, plus TPCs never used for clusters): sizes "
+          f"{R['gpc_map']['sizes']}; components touched by each group: "
+          f"{R['gpc_map']['gpcs_of_group']}", "",
+          "## Single groups (inside one sub-reach window)", "", "| group | SMs | GB/s |", "|---|---|---|"]
+    for s in R["single_groups"]:
+        L.append(f"| {s['group']} | {s['sms']} | {s['gbps']:.0f} |")
+    ratios = [x["ratio_to_sum_of_singles"] for x in R["group_pairs_distinct_windows"]]
+    if ratios:
+        L += ["", f"group pairs in distinct windows / sum of the two singles: min {min(ratios):.3f} "
+                  f"median {float(np.median(ratios)):.3f} max {max(ratios):.3f} "
+                  f"({len(ratios)} pairs)"]
+    L += ["", "## Grouped windows over the whole buffer", ""]
+    for width, d in R["cfg4_grouped"].items():
+        L += [f"### {width} lines: unrestricted over everything {f(d['unrestricted_full'])}", "",
+              "| window | GiB | coverage | grouped | unrestricted inside one window | naive per-SM |",
+              "|---|---|---|---|---|---|"]
+        for name, r in d["windows"].items():
+            L.append(f"| {name} | {r['window_gib']:.1f} | {r['coverage']:.2f} | {f(r['grouped'])} | "
+                     f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} |")
+        L.append("")
+    L.append(f"total {R['seconds']:.0f} s")
+    return "\n".join(L) + "\n"
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default="gpurun_out/report")
+    ap.add_argument("--quick", action="store_true")
+    a = ap.parse_args(argv)
+    R = run(Path(a.out), a.quick)
+    print(markdown(R))
+    return 0
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())

@@ -1,0 +1,165 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times: one
+buffer of ~90 % of free HBM, 32 warps on every SM, 2^8 x 64 reads per warp; outputs the oracle can
+compute one by one are sampled (every 37th warp, the first and the last)."""
+import numpy as np
+import pytest
+
+import oracle
+import rr_inputs
+from paper_2405_11425_b200 import binding as rr
+from paper_2405_11425_b200 import build as rr_build
+from paper_2405_11425_b200.pipeline import Session
+
+pytestmark = pytest.mark.gpu
+GiB = 1 << 30
+WPS = 32
+
+
+@pytest.fixture(scope="module")
+def ses():
+    import torch
+    rr_build.build()
+    torch.cuda.set_device(0)
+    torch.cuda.empty_cache()
+    s = Session(frac_of_free=0.90)
+    assert s.region_bytes > 100 * GiB, "these tests are meant for a GPU with its HBM free"
+    rate = s.fill()
+    assert rate > 100
+    yield s
+    del s.buf
+    torch.cuda.empty_cache()
+
+
+def _sample(n):
+    return sorted(set(list(range(0, n, 37)) + [0, n - 1]))
+
+
+def _check_sampled(ses, got, region, W, reads, seed, groups=None, windows=None, first=0):
+    V = ses.nsm * WPS
+    L = region // (128 * W)
+    for v in _sample(V):
+        sm = v // WPS
+        base, n = 0, L
+        if groups is not None:
+            if groups[sm] == 0xFFFF:
+                assert tuple(got[v]) == (0, 0)
+                continue
+            base, n = map(int, windows[groups[sm]])
+        assert tuple(got[v]) == oracle.warp_checksum(seed, v, first, reads, W, base, n), (v, W)
+
+
+def test_fill_of_the_whole_buffer_sampled_beyond_32_bit_indices(ses):
+    words = ses.buf.view(ses.torch.int32)
+    n = ses.region_bytes // 4
+    assert n > 1 << 32                                     # word indices need 64 bits
+    rng = np.random.default_rng(1)
+    starts = [0, (1 << 32) - 2048, (1 << 32), (1 << 33) + 5, n - 4096]
+    starts += [int(x) for x in rng.integers(0, n - 4096, 24)]
+    for s in starts:
+        got = words[s:s + 4096].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, oracle.fill(s, 4096)), s
+
+
+@pytest.mark.parametrize("size_gib", list(rr_inputs.CFG1_SIZES_GIB) + [None])
+def test_cfg1_unrestricted_sizes_sampled(ses, size_gib):
+    region = ses.region_bytes if size_gib is None else size_gib * GiB
+    if region > ses.region_bytes:
+        pytest.skip("buffer smaller than this sweep point")
+    reads = rr_inputs.CFG1_READS_PER_ITER * 4
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=reads, seed=rr_inputs.CFG1_SEED)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == ses.nsm and res.bytes == ses.nsm * WPS * reads * 128
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), region, 1, reads, rr_inputs.CFG1_SEED)
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+def test_cfg2_widths_at_32_gib_sampled(ses, W):
+    reads = 1024
+    p = ses.params(rr_inputs.CFG2_REGION, W=W, warps_per_sm=WPS, reads_per_warp=reads,
+                   seed=rr_inputs.CFG2_SEED)
+    rr.rr_random_read(p, ses.out, ses.scratch)
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), rr_inputs.CFG2_REGION, W, reads,
+                   rr_inputs.CFG2_SEED)
+
+
+@pytest.mark.parametrize("W", [1, 2])
+def test_cfg4_bench_launch_configuration_sampled(ses, W):
+    # what bench.py times: whole buffer, 24 SM groups, windows of 35 GiB, 16384 reads per warp,
+    # continuing the stream at a later first_read
+    region = ses.region_bytes
+    groups = rr_inputs.synthetic_group_map(ses.nsm, 24, seed=7)
+    windows, cov = rr.rr_make_windows(region, W, 35 * GiB, 24)
+    assert cov == 1.0
+    reads, first = 256 * 64, 256 * 64 * 3
+    p = ses.params(region, W=W, warps_per_sm=WPS, reads_per_warp=reads, first_read=first,
+                   seed=rr_inputs.CFG4_SEED, group_of_sm=groups, windows=windows)
+    assert rr.rr_random_read(p, ses.out, ses.scratch, timed=False) is None   # as bench launches it
+    rep = rr.rr_read_report(p, ses.scratch)
+    assert rep.sms_covered == ses.nsm and rep.bytes == ses.nsm * WPS * reads * 128 * W
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), region, W, reads, rr_inputs.CFG4_SEED,
+                   groups, windows, first)
+
+
+def test_cfg4_naive_control_and_inactive_sms_sampled(ses):
+    region = ses.region_bytes
+    win, cov = rr.rr_make_windows(region, 1, region // 2, ses.nsm, policy=1, seed=23)
+    groups = np.arange(ses.nsm, dtype=np.uint16)
+    groups[5::11] = 0xFFFF
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=512, seed=23,
+                   group_of_sm=groups, windows=win)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == int((groups != 0xFFFF).sum())
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), region, 1, 512, 23, groups, win)
+
+
+def test_cfg3_probe_over_the_whole_buffer(ses):
+    total = 1 << 18
+    per_warp = total // 2 // WPS
+    a, b = 2, ses.nsm - 3
+    res = rr.rr_probe_pair(ses.buf, ses.region_bytes, a, b, total, WPS, rr_inputs.CFG3_SEED,
+                           ses.probe_out, ses.scratch)
+    got = ses.probe_out.cpu().numpy().view(np.uint32)
+    L = ses.region_bytes // 128
+    for w in (0, 7, 31):
+        assert tuple(got[w]) == oracle.warp_checksum(rr_inputs.CFG3_SEED, a * WPS + w, 0, per_warp,
+                                                     1, 0, L)
+        assert tuple(got[WPS + w]) == oracle.warp_checksum(rr_inputs.CFG3_SEED, b * WPS + w, 0,
+                                                           per_warp, 1, 0, L)
+    assert res.bytes == total * 128 and res.gbps > 1
+
+
+def test_stride_mode_covers_every_line_of_a_large_prefix_once(ses):
+    # property that holds at any size: with V*R == L every line is read once, so the per-warp
+    # sums add up to the sum of the region's words, which the oracle can fold in chunks
+    V = ses.nsm * WPS
+    R = 2048
+    region = V * R * 128                                     # ~1.2 GiB
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=R,
+                   index_mode=rr.RR_INDEX_STRIDE)
+    rr.rr_random_read(p, ses.out, ses.scratch)
+    got = ses.checksums(V)
+    x, s = 0, 0
+    step = 1 << 24
+    for first in range(0, region // 4, step):
+        w = oracle.fill(first, min(step, region // 4 - first))
+        x ^= int(np.bitwise_xor.reduce(w))
+        s = (s + int(w.astype(np.uint64).sum())) & 0xFFFFFFFF
+    assert int(np.bitwise_xor.reduce(got[:, 0])) == x
+    assert int(got[:, 1].astype(np.uint64).sum() & 0xFFFFFFFF) == s
+
+
+def test_contention_groups_nest_inside_gpcs(ses):
+    # two independent views of the layout: timing (pair probe beyond the reach + clustering) and
+    # cluster placement (no timing).  Every contention group must lie inside one GPC; TPCs that
+    # the cluster scheduler never places a multi-block cluster on (components of one TPC) carry
+    # no GPC information and are left out of the comparison.
+    groups = ses.discover_groups(total_reads=1 << 16, repeats=3)
+    assert groups.n_groups >= 2 and groups.confidence > 4.0
+    assert np.array_equal(groups.group_of_sm[0::2], groups.group_of_sm[1::2])   # TPC mates together
+    gpc, n_gpcs = rr.rr_gpc_map(ses.scratch, ses.nsm)
+    informative = np.bincount(gpc)[gpc] > 2
+    for k in range(groups.n_groups):
+        members = (groups.group_of_sm == k) & informative
+        assert len(set(gpc[members].tolist())) <= 1, (k, np.where(groups.group_of_sm == k)[0])
+    # and the partition is finer than the GPCs, as the paper found on its card
+    assert groups.n_groups > int((np.bincount(gpc) > 2).sum())

@@ -247,3 +247,16 @@ def test_cluster_two_sms_and_ties(dev):
     g, G, conf, h = rr.rr_cluster(T, dev.scratch)
     og, oG, oconf, oh = oracle.cluster(T)
     assert G == oG == 1 and np.array_equal(h, oh)
+
+
+def test_gpc_map_from_cluster_placement(dev):
+    g, n_gpcs = rr.rr_gpc_map(dev.scratch, dev.nsm)
+    assert g.shape == (dev.nsm,) and g.min() == 0 and g.max() == n_gpcs - 1
+    assert 2 <= n_gpcs <= dev.nsm // 2
+    assert np.array_equal(g[0::2], g[1::2])            # the two SMs of a TPC share a GPC
+    firsts = [int(np.argmax(g == k)) for k in range(n_gpcs)]
+    assert firsts == sorted(firsts)                    # canonical labels
+    g2, n2 = rr.rr_gpc_map(dev.scratch, dev.nsm)
+    assert n2 == n_gpcs and np.array_equal(g, g2)      # placement facts, not timing: repeatable
+    with pytest.raises(rr.RRError):
+        rr.rr_gpc_map(dev.scratch, dev.nsm + 1)

@@ -17,8 +17,6 @@ FAKE = 0x7F0000000000
 def test_requests_beyond_the_built_in_scratch_are_refused_before_any_launch():
     rr_build.build()
     lib = rr._load()
-    p = rr.ReadParams(FAKE, 1 << 20, warps_per_sm=64, reads_per_warp=4)
-    assert lib.rr_random_read_static(ctypes.byref(p.c), FAKE, None, 0) == rr.RR_ERR_STATIC_LIMIT
     g = np.zeros(200, np.uint16)
     p = rr.ReadParams(FAKE, 1 << 20, warps_per_sm=8, reads_per_warp=4, nsm=200, group_of_sm=g,
                       windows=[[0, 8]])
