@@ -196,11 +196,15 @@ def run_gpu(args):
     peaks, peak_kind = _peaks()
 
     # ---- calibration (untimed): fill, groups, reach, windows --------------------------------
+    t_cal = time.time()
     ses = Session()
     fill_gbps = ses.fill()
     fill_gbps = max(fill_gbps, ses.fill())
     groups = ses.discover_groups(total_reads=args.probe_reads, repeats=args.probe_repeats)
+    gpc, n_gpc = rr.rr_gpc_map(ses.scratch, ses.nsm)
+    t_reach = time.time()
     reach = ses.measure_reach()
+    t_reach = time.time() - t_reach
     N = ses.region_bytes
     unrestricted_full, _ = ses.read(N, seed=SEED, reads_per_warp=READS_PER_ITER * 16)
     if reach.cliff:
@@ -222,6 +226,11 @@ def run_gpu(args):
     ctrl_groups, ctrl_win, _ = ses.naive_control(S, SEED)
     naive_control, _ = ses.read(N, seed=SEED, reads_per_warp=READS_PER_ITER * 16,
                                 group_of_sm=ctrl_groups, windows=ctrl_win)
+    win256, _ = ses.windows(groups, S, W=2)
+    grouped_256, _ = ses.read(N, W=2, seed=SEED, reads_per_warp=READS_PER_ITER * 16,
+                              group_of_sm=groups.group_of_sm, windows=win256)
+    unrestricted_256, _ = ses.read(N, W=2, seed=SEED, reads_per_warp=READS_PER_ITER * 16)
+    t_cal = time.time() - t_cal
 
     # ---- timed region: device-resident, asynchronous launches -------------------------------
     reads = READS_PER_ITER * ITERS_PER_STEP
@@ -321,18 +330,23 @@ def run_gpu(args):
             "parity": parity,
             "calibration": {
                 "device": ses.info["name"], "uuid": ses.info["uuid"], "nsm": ses.nsm,
+                "seconds_total": t_cal, "seconds_reach_sweep": t_reach,
                 "fill_gbps": fill_gbps,
                 "probe": {"seconds": groups.probe_seconds, "pairs": ses.nsm * (ses.nsm + 1) // 2,
                           "reads_per_pair": args.probe_reads, "repeats": args.probe_repeats,
                           "overlap_min": groups.overlap_min},
                 "groups": {"n": groups.n_groups, "confidence": groups.confidence,
-                           "sizes": groups.sizes, "group_of_sm": groups.group_of_sm.tolist()},
+                           "sizes": groups.sizes, "group_of_sm": groups.group_of_sm.tolist(),
+                           "cluster_placement_components": np.bincount(gpc).tolist(),
+                           "components_of_group": [sorted(set(gpc[groups.group_of_sm == k].tolist()))
+                                                   for k in range(groups.n_groups)]},
                 "reach": {"cliff": reach.cliff, "plateau_gbps": reach.plateau_gbps,
                           "reach_gib": reach.reach_bytes / GiB,
                           "sweep": [[s / GiB, g] for s, g in reach.sweep]},
                 "unrestricted_full_gbps": unrestricted_full,
                 "unrestricted_in_window_gbps": in_window,
                 "naive_per_sm_control_gbps": naive_control,
+                "grouped_256B_gbps": grouped_256, "unrestricted_full_256B_gbps": unrestricted_256,
                 "window_sweep": window_sweep,
             },
         }

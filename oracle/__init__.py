@@ -67,6 +67,10 @@ def _load():
         lib.orc_read_per_sm.argtypes = [u64, u32, u32, u32, u32, u64, u64, u64, p, p, p, u32, p]
         lib.orc_make_windows.restype = i32
         lib.orc_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p, p]
+        lib.orc_make_weighted_windows.restype = i32
+        lib.orc_make_weighted_windows.argtypes = [u64, u32, u32, p, u64, u64, p, p, p]
+        lib.orc_read_pooled.restype = i32
+        lib.orc_read_pooled.argtypes = [u64, u32, u32, p, p, p, u64, u64, u64, p]
         lib.orc_cluster.restype = i32
         lib.orc_cluster.argtypes = [p, u32, u32, p, p, p, p]
         lib.orc_reach.restype = i32
@@ -167,6 +171,40 @@ def make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int, po
     if rc != 0:
         raise OracleError(rc)
     return np.stack([wb, wn], axis=1), float(cov.value)
+
+
+def make_weighted_windows(region_bytes: int, W: int, weights, n_warps: int,
+                          max_window_bytes: int = 0):
+    """Windows and logical-warp ranges in proportion to integer group weights.
+
+    Returns ((G, 2) uint32 {base_line, n_lines}, warp_start uint32[G+1])."""
+    w = np.ascontiguousarray(weights, dtype=np.uint32)
+    G = int(w.shape[0])
+    wb = np.zeros(G, dtype=np.uint32)
+    wn = np.zeros(G, dtype=np.uint32)
+    ws = np.zeros(G + 1, dtype=np.uint32)
+    rc = _load().orc_make_weighted_windows(region_bytes, W, G, _ptr(w), n_warps, max_window_bytes,
+                                           _ptr(wb), _ptr(wn), _ptr(ws))
+    if rc != 0:
+        raise OracleError(rc)
+    return np.stack([wb, wn], axis=1), ws
+
+
+def read_pooled(region_bytes: int, W: int, windows, warp_start, reads: int, seed: int,
+                first_read: int = 0) -> np.ndarray:
+    """Checksums of logical warps 0..warp_start[-1]-1, each inside its group's window."""
+    w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+    wb = np.ascontiguousarray(w[:, 0])
+    wn = np.ascontiguousarray(w[:, 1])
+    ws = np.ascontiguousarray(warp_start, dtype=np.uint32)
+    if ws.shape != (w.shape[0] + 1,):
+        raise OracleError(-1)
+    out = np.zeros((int(ws[-1]), 2), dtype=np.uint32)
+    rc = _load().orc_read_pooled(region_bytes, W, w.shape[0], _ptr(wb), _ptr(wn), _ptr(ws),
+                                 first_read, reads, seed, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
 
 
 def cluster(T, solo_normalise: bool = False):

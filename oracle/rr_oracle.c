@@ -215,6 +215,78 @@ int32_t orc_make_windows(uint64_t region_bytes, uint32_t W, uint64_t window_byte
     return ORC_OK;
 }
 
+/* ---- O4b: windows and work in proportion to each group's capacity ----------------
+ * Section 2.3 runs every resource group on its own and finds that a group's throughput
+ * is a property of the group.  If every SM does the same work, the groups with the most
+ * SMs per unit of capacity finish last and set the time.  Reading: give group g the
+ * integer weight w_g (its measured solo throughput); with P_g = w_0 + .. + w_(g-1) and
+ * T = P_G, group g owns
+ *   lines  [floor(L * P_g / T), floor(L * P_(g+1) / T))   -- windows tile the region
+ *   warps  [floor(V * P_g / T), floor(V * P_(g+1) / T))   -- logical warps, same rule
+ * so reads stay uniformly dense over the region and each group's share of the work
+ * matches its share of the capacity.  warp_start receives G+1 entries.
+ * Errors: a group left without lines or without warps, or a window above max_window_bytes
+ * (0 = no limit).                                                                  */
+int32_t orc_make_weighted_windows(uint64_t region_bytes, uint32_t W, uint32_t n_groups,
+                                  const uint32_t *weight, uint64_t n_warps,
+                                  uint64_t max_window_bytes, uint32_t *win_base,
+                                  uint32_t *win_n, uint32_t *warp_start)
+{
+    if (!orc_width_ok(W) || n_groups == 0 || !weight || !win_base || !win_n || !warp_start ||
+        n_warps == 0 || n_warps > 0xFFFFFFFFull)
+        return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    uint64_t T = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        if (weight[g] == 0) return ORC_ERR_ARG;
+        T += weight[g];
+    }
+    if (T > 0xFFFFFFFFull) return ORC_ERR_RANGE; /* keeps L*P and V*P inside 64 bits */
+    uint64_t P = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        uint64_t lo = L * P / T, hi = L * (P + weight[g]) / T;
+        uint64_t vlo = n_warps * P / T, vhi = n_warps * (P + weight[g]) / T;
+        if (hi == lo || vhi == vlo) return ORC_ERR_RANGE;
+        if (max_window_bytes && (hi - lo) * 128ull * W > max_window_bytes) return ORC_ERR_RANGE;
+        win_base[g] = (uint32_t)lo;
+        win_n[g] = (uint32_t)(hi - lo);
+        warp_start[g] = (uint32_t)vlo;
+        P += weight[g];
+    }
+    warp_start[n_groups] = (uint32_t)n_warps;
+    return ORC_OK;
+}
+
+/* Pooled mode: logical warps v = 0 .. V-1 (V = warp_start[G]); warp v belongs to the group
+ * g with warp_start[g] <= v < warp_start[g+1] and reads inside that group's window.
+ * Which SM performs which of its reads is left to the machine; the checksums do not
+ * depend on it.  out holds V pairs {X, S}.                                          */
+int32_t orc_read_pooled(uint64_t region_bytes, uint32_t W, uint32_t n_groups,
+                        const uint32_t *win_base, const uint32_t *win_n,
+                        const uint32_t *warp_start, uint64_t first_read, uint64_t reads,
+                        uint64_t seed, uint32_t *out)
+{
+    if (!orc_width_ok(W) || n_groups == 0 || !win_base || !win_n || !warp_start || !out)
+        return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    if (warp_start[0] != 0) return ORC_ERR_ARG;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        if (warp_start[g + 1] < warp_start[g]) return ORC_ERR_ARG;
+        if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
+    }
+    uint64_t V = warp_start[n_groups];
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        int64_t lo = warp_start[g], hi = warp_start[g + 1];
+#pragma omp parallel for schedule(dynamic, 16)
+        for (int64_t v = lo; v < hi; ++v)
+            orc_warp_checksum(ORC_INDEX_RANDOM, seed, (uint64_t)v, V, first_read, reads, W,
+                              win_base[g], win_n[g], &out[2 * v], &out[2 * v + 1]);
+    }
+    return ORC_OK;
+}
+
 /* ---- O5: SM x SM matrix -> groups (Section 2.2, Figures 2 and 3) ---------------
  * 1. symmetrise off-diagonal entries in double: t = (T_ij + T_ji) / 2; with flag
  *    ORC_CLUSTER_SOLO_NORMALISE, divide by the two SMs' solo rates on the diagonal:

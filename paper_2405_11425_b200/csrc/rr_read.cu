@@ -461,6 +461,7 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     auto cleanup = [&]() {
         if (e0) cudaEventDestroy(e0);
         if (e1) cudaEventDestroy(e1);
+        e0 = e1 = nullptr;
     };
 #define RR_CUDA_C(call)                        \
     do {                                       \
