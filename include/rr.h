@@ -60,10 +60,13 @@ extern "C" {
 /* ---- enums (plain integers in the structs) ---- */
 #define RR_MODE_LOGICAL 0u /* v = global warp index 0..n_warps-1, window = whole region        */
 #define RR_MODE_PER_SM 1u  /* v = smid * warps_per_sm + warp, window by SM group               */
+#define RR_MODE_POOLED 2u  /* logical warps owned by SM groups; the group's SMs share the work  */
 #define RR_INDEX_RANDOM 0u
 #define RR_INDEX_STRIDE 1u
 #define RR_VARIANT_LDG 0u         /* ld.global.nc.L1::no_allocate vector loads                  */
 #define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
+#define RR_VARIANT_PACKED 2u      /* every lane loads 16 bytes: one warp load covers 4/W lines  */
+                                  /* (same lines and words; fewer instructions per line)        */
 
 const char *rr_strerror(int32_t code);
 const char *rr_last_cuda_error(void);
@@ -112,9 +115,22 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   Otherwise group_of_sm[nsm] (HOST) gives each SM's group or RR_SM_INACTIVE, and
  *   windows[n_groups] (HOST) the window of each group.  out has nsm*warps_per_sm entries;
  *   inactive SMs' entries are {0,0}.  nsm must equal the device's SM count (0 = take it).
+ * RR_MODE_POOLED (Section 2.3 shows that a group's throughput belongs to the group, not to its
+ *   SMs): n_warps logical warps; group g owns warps warp_start[g] .. warp_start[g+1]-1 (HOST
+ *   array of n_groups+1 entries, warp_start[0] = 0, warp_start[n_groups] = n_warps) and they
+ *   read inside windows[g].  The group's work is the line of its warps' reads; the persistent
+ *   blocks of the group's SMs (warps_per_sm physical warps each) grab runs of that line from a
+ *   per-group counter -- long runs at first, never shorter than pool_block_reads at the end --
+ *   until it is used up.  A group with more SMs then does not do more work than its shared
+ *   translation path can carry, and no group becomes the straggler when warp_start follows the
+ *   groups' capacities (rr_make_weighted_windows).  out has n_warps entries, accumulated with
+ *   atomics (the call clears it first); the checksums do not depend on which SM did what.
+ *   Every group that owns warps needs at least one active SM, else RR_ERR_MAP.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
- * unroll: independent loads kept in flight per warp: 0 (= default) or 2, 4, 8, 16.
+ * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
+ *   so that unroll * W <= 32 (the ring lives in registers).  RR_VARIANT_PACKED counts warp
+ *   loads of 4/W lines each (1, 2, 4 or 8; default 4).
  *
  * out_dev (DEVICE, 8-byte aligned): pairs {X, S} of uint32.  scratch_dev: rr_scratch_bytes().
  * res == NULL: asynchronous on `stream`, no timing; decode the scratch later with
@@ -130,9 +146,9 @@ typedef struct {
     uint32_t words_per_lane;    /* W: 1, 2, 4                                                  */
     uint32_t mode;              /* RR_MODE_*                                                   */
     uint32_t index_mode;        /* RR_INDEX_*                                                  */
-    uint32_t n_warps;           /* LOGICAL                                                     */
-    uint32_t warps_per_sm;      /* PER_SM: 1..RR_MAX_WARPS_PER_SM (one block per SM)           */
-    uint32_t nsm;               /* PER_SM: SM count of the device, 0 = query                   */
+    uint32_t n_warps;           /* LOGICAL, POOLED: number of logical warps                    */
+    uint32_t warps_per_sm;      /* PER_SM, POOLED: 1..RR_MAX_WARPS_PER_SM (one block per SM)   */
+    uint32_t nsm;               /* PER_SM, POOLED: SM count of the device, 0 = query           */
     uint64_t reads_per_warp;
     uint64_t first_read;
     uint64_t seed;
@@ -141,13 +157,14 @@ typedef struct {
     uint32_t n_groups;
     uint32_t variant;           /* RR_VARIANT_*                                                */
     uint32_t unroll;
-    uint32_t reserved;          /* must be 0                                                   */
+    uint32_t pool_block_reads;  /* POOLED: smallest grab in reads, 0 = 64; else must be 0      */
+    const uint32_t *warp_start; /* POOLED: HOST [n_groups+1]; else NULL                        */
 } rr_read_params_t;
 
 typedef struct {
     double seconds_event;   /* CUDA events around the launch (0 when not timed)                */
     double seconds_device;  /* max block end - min block start, %globaltimer                   */
-    uint64_t bytes;         /* active warps * reads_per_warp * 128 * W                         */
+    uint64_t bytes;         /* (active or logical) warps * reads_per_warp * 128 * W            */
     double gbps;            /* bytes / seconds_event / 1e9 (seconds_device when not timed)     */
     uint32_t status;        /* device status word: 0 = clean                                   */
     uint32_t violations;    /* checked variant: addresses rejected                             */
@@ -165,6 +182,13 @@ int32_t rr_random_read(const rr_read_params_t *params /*HOST*/, void *out_dev /*
 int32_t rr_read_report(const rr_read_params_t *params /*HOST*/, const void *scratch_dev,
                        rr_result_t *res /*HOST*/, void *stream);
 
+/* Start and end of every SM's block in the last rr_random_read that used this scratch
+ * (%globaltimer, ns; both 0 for an SM that ran no block).  RR_MODE_PER_SM / RR_MODE_POOLED only.
+ * t_start_host, t_end_host: HOST [nsm].  Synchronises `stream` first.  With these a caller can
+ * see which SM group finished last and shift work between groups (Section 2.3).               */
+int32_t rr_read_block_times(const void *scratch_dev /*DEVICE*/, uint32_t nsm,
+                            uint64_t *t_start_host, uint64_t *t_end_host, void *stream);
+
 /* ---- random line reads for callers that cannot allocate device memory ----------------------
  * (The paper has no counterpart: this is a packaging variant of rr_random_read.)
  *
@@ -177,8 +201,9 @@ int32_t rr_read_report(const rr_read_params_t *params /*HOST*/, const void *scra
  * until the process exits).  It calls no allocation routine of any kind, and creates no events:
  * res->seconds_event is 0 and res->gbps is computed from the device-side timers.
  *
- * Limit: at most RR_STATIC_MAX_SM SMs (the device's count, or the nsm passed in); a larger
- * count returns RR_ERR_STATIC_LIMIT before launching.  All other arguments, outputs and
+ * Limit: at most RR_STATIC_MAX_SM SMs (the device's count, or the nsm passed in), and no
+ * RR_MODE_POOLED (its work counters do not fit); both return RR_ERR_STATIC_LIMIT before
+ * launching.  All other arguments, outputs and
  * status codes are those of rr_random_read (the caller still passes buf and out_dev).
  *
  * The first call on each device looks up the device address of the built-in array (the device
@@ -259,6 +284,21 @@ int32_t rr_gpc_map(void *scratch_dev /*DEVICE*/, int32_t *gpc_of_sm_host /*HOST*
 int32_t rr_make_windows(uint64_t region_bytes, uint32_t words_per_lane, uint64_t window_bytes,
                         uint32_t n_groups, uint32_t policy, uint64_t seed,
                         rr_window_t *out_host /*HOST n_groups*/, double *coverage);
+
+/* ---- windows and work in proportion to each group's capacity (host only) ---------------------
+ * Paper, Section 2.3 (each resource group run on its own): on B200 a group's throughput is capped
+ * by its shared translation path whatever its SM count, so equal work per SM makes the largest
+ * groups finish last.  Given an integer weight per group (its measured solo GB/s, say), with
+ * P_g = w_0 + .. + w_(g-1) and T = P_G, group g gets
+ *   lines [floor(L*P_g/T), floor(L*P_(g+1)/T))      (windows tile the region, uniform density)
+ *   warps [floor(V*P_g/T), floor(V*P_(g+1)/T))      (V = n_warps logical warps)
+ * for use with RR_MODE_POOLED.  warp_start_host receives n_groups+1 entries.  RR_ERR_RANGE if a
+ * group is left without lines or warps, the weights sum above 2^32-1, or a window exceeds
+ * max_window_bytes (0 = no limit; pass the measured reach).                                    */
+int32_t rr_make_weighted_windows(uint64_t region_bytes, uint32_t words_per_lane, uint32_t n_groups,
+                                 const uint32_t *weight_host, uint32_t n_warps,
+                                 uint64_t max_window_bytes, rr_window_t *out_host,
+                                 uint32_t *warp_start_host);
 
 /* ---- A8: plateau, cliff and reach from a size sweep (host only) ----------------------------
  * Paper, Section 2.1 / Figure 1 ("something dramatic happens when the memory region is larger

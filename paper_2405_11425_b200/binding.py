@@ -21,15 +21,16 @@ RR_ERR_SM_UNCOVERED, RR_ERR_TIMEOUT, RR_ERR_CHECK, RR_ERR_UNSUPPORTED = -6, -7, 
 RR_ERR_STATIC_LIMIT = -10
 RR_STATIC_MAX_SM, RR_STATIC_SCRATCH_BYTES = 192, 5888
 RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0xFFFF
-RR_MODE_LOGICAL, RR_MODE_PER_SM = 0, 1
+RR_MODE_LOGICAL, RR_MODE_PER_SM, RR_MODE_POOLED = 0, 1, 2
 RR_INDEX_RANDOM, RR_INDEX_STRIDE = 0, 1
-RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED = 0, 1
+RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED, RR_VARIANT_PACKED = 0, 1, 2
 
 EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
     "rr_random_read", "rr_read_report", "rr_probe_pair", "rr_probe_matrix_scratch_bytes",
     "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach", "rr_random_read_static",
-    "rr_gpc_map",
+    "rr_gpc_map", "rr_make_weighted_windows",
+    "rr_read_block_times",
 )
 
 
@@ -56,7 +57,8 @@ class _ReadParams(ctypes.Structure):
         ("reads_per_warp", ctypes.c_uint64), ("first_read", ctypes.c_uint64),
         ("seed", ctypes.c_uint64), ("group_of_sm", ctypes.c_void_p),
         ("windows", ctypes.c_void_p), ("n_groups", ctypes.c_uint32),
-        ("variant", ctypes.c_uint32), ("unroll", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("variant", ctypes.c_uint32), ("unroll", ctypes.c_uint32),
+        ("pool_block_reads", ctypes.c_uint32), ("warp_start", ctypes.c_void_p),
     ]
 
 
@@ -124,6 +126,8 @@ def _load():
     lib.rr_random_read.argtypes = [p, p, p, p, p]
     lib.rr_random_read_static.restype = i32
     lib.rr_random_read_static.argtypes = [p, p, p, p]
+    lib.rr_read_block_times.restype = i32
+    lib.rr_read_block_times.argtypes = [p, u32, p, p, p]
     lib.rr_read_report.restype = i32
     lib.rr_read_report.argtypes = [p, p, p, p]
     lib.rr_probe_pair.restype = i32
@@ -138,6 +142,8 @@ def _load():
     lib.rr_gpc_map.argtypes = [p, p, p, u32, p]
     lib.rr_make_windows.restype = i32
     lib.rr_make_windows.argtypes = [u64, u32, u64, u32, u32, u64, p, p]
+    lib.rr_make_weighted_windows.restype = i32
+    lib.rr_make_weighted_windows.argtypes = [u64, u32, u32, p, u32, u64, p, p]
     lib.rr_reach.restype = i32
     lib.rr_reach.argtypes = [p, p, u32, p, p]
     _lib = lib
@@ -198,9 +204,13 @@ class ReadParams:
     def __init__(self, buf, region_bytes: int, *, W: int = 1, mode: int = RR_MODE_PER_SM,
                  index_mode: int = RR_INDEX_RANDOM, n_warps: int = 0, warps_per_sm: int = 32,
                  nsm: int = 0, reads_per_warp: int = 0, first_read: int = 0, seed: int = 0,
-                 group_of_sm=None, windows=None, variant: int = RR_VARIANT_LDG, unroll: int = 0):
+                 group_of_sm=None, windows=None, variant: int = RR_VARIANT_LDG, unroll: int = 0,
+                 warp_start=None, pool_block_reads: int = 0):
         self._groups = None
         self._windows = None
+        self._warp_start = None
+        if warp_start is not None:
+            self._warp_start = np.ascontiguousarray(warp_start, dtype=np.uint32)
         n_groups = 0
         if group_of_sm is not None:
             self._groups = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
@@ -213,7 +223,8 @@ class ReadParams:
             reads_per_warp, first_read, seed,
             self._groups.ctypes.data if self._groups is not None else None,
             self._windows.ctypes.data if self._windows is not None else None,
-            n_groups, variant, unroll, 0)
+            n_groups, variant, unroll, pool_block_reads,
+            self._warp_start.ctypes.data if self._warp_start is not None else None)
 
 
 def _result(r: _Result) -> ReadResult:
@@ -247,6 +258,15 @@ def rr_read_report(params: ReadParams, scratch, stream=None) -> ReadResult:
     _check(_load().rr_read_report(ctypes.byref(params.c), _dev(scratch), ctypes.byref(res),
                                   _stream(stream)), "rr_read_report")
     return _result(res)
+
+
+def rr_read_block_times(scratch, nsm: int, stream=None):
+    """(t_start, t_end) uint64[nsm] in ns of every SM's block in the last read on this scratch."""
+    t0 = np.zeros(nsm, dtype=np.uint64)
+    t1 = np.zeros(nsm, dtype=np.uint64)
+    _check(_load().rr_read_block_times(_dev(scratch), nsm, t0.ctypes.data, t1.ctypes.data,
+                                       _stream(stream)), "rr_read_block_times")
+    return t0, t1
 
 
 def rr_probe_pair(buf, region_bytes: int, sm_a: int, sm_b: int, total_reads: int,
@@ -305,6 +325,19 @@ def rr_make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int,
     _check(_load().rr_make_windows(region_bytes, W, window_bytes, n_groups, policy, seed,
                                    out.ctypes.data, ctypes.byref(cov)), "rr_make_windows")
     return out[:n_groups], float(cov.value)
+
+
+def rr_make_weighted_windows(region_bytes: int, W: int, weights, n_warps: int,
+                             max_window_bytes: int = 0):
+    """Returns ((G, 2) uint32 windows, warp_start uint32[G+1]) in proportion to integer weights."""
+    w = np.ascontiguousarray(weights, dtype=np.uint32)
+    G = int(w.shape[0])
+    win = np.zeros((max(G, 1), 2), dtype=np.uint32)
+    ws = np.zeros(G + 1, dtype=np.uint32)
+    _check(_load().rr_make_weighted_windows(region_bytes, W, G, w.ctypes.data, n_warps,
+                                            max_window_bytes, win.ctypes.data, ws.ctypes.data),
+           "rr_make_weighted_windows")
+    return win[:G], ws
 
 
 def rr_reach(size_bytes, gbps):

@@ -2,7 +2,7 @@
 
     python -m paper_2405_11425_b200.cases read  [--region-gib 4] [--W 1] [--reads 4096]
                                                 [--launches 3] [--groups 0] [--unroll 0]
-                                                [--stride] [--warps-per-sm 32]
+                                                [--stride] [--warps-per-sm 32] [--packed] [--pooled]
     python -m paper_2405_11425_b200.cases fill  [--region-gib 4] [--launches 3]
     python -m paper_2405_11425_b200.cases probe [--region-gib 4] [--reads 65536] [--pairs 4]
     python -m paper_2405_11425_b200.cases cluster [--n 148]
@@ -31,6 +31,9 @@ def main(argv=None):
     ap.add_argument("--groups", type=int, default=0, help="synthetic SM groups, one window each")
     ap.add_argument("--unroll", type=int, default=0)
     ap.add_argument("--stride", action="store_true")
+    ap.add_argument("--packed", action="store_true", help="16-byte lanes, 4/W lines per warp load")
+    ap.add_argument("--pooled", action="store_true",
+                    help="logical warps owned by the synthetic groups, work shared inside a group")
     ap.add_argument("--warps-per-sm", type=int, default=32)
     ap.add_argument("--pairs", type=int, default=4)
     ap.add_argument("--n", type=int, default=148)
@@ -85,9 +88,22 @@ def main(argv=None):
         groups = rr_inputs.synthetic_group_map(nsm, a.groups, seed=1)
         windows, _ = rr.rr_make_windows(region, a.W, -(-region // a.groups), a.groups)
     o = torch.zeros((nsm * a.warps_per_sm, 2), dtype=torch.int32, device="cuda")
-    p = rr.ReadParams(buf, region, W=a.W, warps_per_sm=a.warps_per_sm, reads_per_warp=a.reads,
-                      seed=7, unroll=a.unroll, group_of_sm=groups, windows=windows,
-                      index_mode=rr.RR_INDEX_STRIDE if a.stride else rr.RR_INDEX_RANDOM)
+    variant = rr.RR_VARIANT_PACKED if a.packed else rr.RR_VARIANT_LDG
+    if a.pooled:
+        import rr_inputs
+        n_groups = a.groups or 24
+        groups = rr_inputs.synthetic_group_map(nsm, n_groups, seed=1)
+        n_warps = nsm * a.warps_per_sm
+        windows, warp_start = rr.rr_make_weighted_windows(region, a.W, [1] * n_groups, n_warps)
+        p = rr.ReadParams(buf, region, W=a.W, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
+                          warps_per_sm=a.warps_per_sm, nsm=nsm, reads_per_warp=a.reads, seed=7,
+                          unroll=a.unroll, group_of_sm=groups, windows=windows,
+                          warp_start=warp_start, variant=variant)
+    else:
+        p = rr.ReadParams(buf, region, W=a.W, warps_per_sm=a.warps_per_sm, reads_per_warp=a.reads,
+                          seed=7, unroll=a.unroll, group_of_sm=groups, windows=windows,
+                          variant=variant,
+                          index_mode=rr.RR_INDEX_STRIDE if a.stride else rr.RR_INDEX_RANDOM)
     for _ in range(a.launches):
         res = rr.rr_random_read(p, o, scratch)
     out.update(region_bytes=region, W=a.W, reads=a.reads, bytes=res.bytes, gbps=res.gbps,

@@ -130,6 +130,39 @@ extern "C" int32_t rr_make_windows(uint64_t region_bytes, uint32_t W, uint64_t w
     return RR_OK;
 }
 
+extern "C" int32_t rr_make_weighted_windows(uint64_t region_bytes, uint32_t W, uint32_t n_groups,
+                                            const uint32_t *weight, uint32_t n_warps,
+                                            uint64_t max_window_bytes, rr_window_t *out,
+                                            uint32_t *warp_start)
+{
+    if (!(W == 1 || W == 2 || W == 4) || n_groups == 0 || n_groups > RR_MAX_GROUPS || !weight ||
+        !out || !warp_start || n_warps == 0)
+        return RR_ERR_ARG;
+    const uint64_t line = 128ull * W;
+    const uint64_t L = region_bytes / line;
+    if (L == 0 || L > 0xFFFFFFFFull) return RR_ERR_RANGE;
+    uint64_t total = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        if (weight[g] == 0) return RR_ERR_ARG;
+        total += weight[g];
+    }
+    if (total > 0xFFFFFFFFull) return RR_ERR_RANGE;  // L * prefix and V * prefix stay in 64 bits
+    uint64_t prefix = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        const uint64_t next = prefix + weight[g];
+        const uint64_t lo = L * prefix / total, hi = L * next / total;
+        const uint64_t vlo = (uint64_t)n_warps * prefix / total, vhi = (uint64_t)n_warps * next / total;
+        if (hi == lo || vhi == vlo) return RR_ERR_RANGE;
+        if (max_window_bytes && (hi - lo) * line > max_window_bytes) return RR_ERR_RANGE;
+        out[g].base_line = (uint32_t)lo;
+        out[g].n_lines = (uint32_t)(hi - lo);
+        warp_start[g] = (uint32_t)vlo;
+        prefix = next;
+    }
+    warp_start[n_groups] = n_warps;
+    return RR_OK;
+}
+
 extern "C" int32_t rr_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
                             double *plateau, uint64_t *reach_bytes)
 {

@@ -34,6 +34,7 @@ struct ScratchHeader {
     uint32_t claim[RR_MAX_SM];
     BlockRecord rec[kMaxRecords];
     ProbeRecord probe;
+    unsigned long long pool_next[RR_MAX_GROUPS];  // POOLED: next work item of each group
 };
 
 // Bytes after the header used by rr_cluster (see rr_cluster.cu).

@@ -20,6 +20,7 @@ namespace rr {
 struct Tables {
     uint16_t group_of_sm[RR_MAX_SM];
     rr_window_t windows[RR_MAX_GROUPS];
+    uint32_t warp_start[RR_MAX_GROUPS + 1];  // POOLED
 };
 
 struct ReadArgs {
@@ -33,12 +34,15 @@ struct ReadArgs {
     uint32_t wps, wpc, cps;  // warps per SM, per block; blocks per SM
     uint32_t nsm;
     uint32_t n_groups;  // 0 = ungrouped
+    uint32_t pool_block;  // POOLED: smallest grab, in reads
     uint2 *out;
     ScratchHeader *scratch;
 };
 
+constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2;
+
 template <int W, int U, bool CHECKED>
-__device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
+__device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, uint64_t region_bytes,
                                            uint64_t key, uint32_t index_mode, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
@@ -119,17 +123,183 @@ __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_
     S = s;
 }
 
-template <int W, int U, bool CHECKED>
+// Packed shape: every lane always loads 16 bytes, so one warp load covers P = 4/W different
+// lines (8 lanes per 128-byte line, 16 per 256-byte line).  Same lines, same words, a quarter
+// (half) of the load, shuffle and address instructions per line -- which matters because this
+// workload runs into the board's power limit and every instruction not issued buys clock.
+template <int W, int U>
+__device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, uint64_t key,
+                                                  uint32_t index_mode, uint64_t v, uint64_t V,
+                                                  uint64_t first, uint64_t reads, uint32_t base,
+                                                  uint32_t n, uint32_t lane, uint32_t &X,
+                                                  uint32_t &S)
+{
+    constexpr int P = 4 / W;     // lines per warp load
+    constexpr int NL = 32 / P;   // warp loads per batch of 32 reads = lanes per line
+    static_assert(W == 1 || W == 2, "16-byte lanes already cover a 512-byte line");
+    static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a batch");
+    const Divisor div = make_divisor(n);
+    const uint32_t sub = lane / NL;  // which of the P lines of a load this lane serves
+    const char *lane_ptr = buf + (lane % NL) * 16u;
+    uint32_t d[U][4];
+    uint32_t x = 0, s = 0;
+
+    auto gen = [&](uint64_t i) -> uint32_t {
+        uint64_t r = (index_mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        return base + mod_exact(r, div);
+    };
+    auto issue = [&](uint32_t line, uint32_t(&dst)[4]) {
+        load_lane<4>(lane_ptr + (uint64_t)line * (128u * W), dst);
+    };
+    auto clear = [&](uint32_t(&dst)[4]) { dst[0] = dst[1] = dst[2] = dst[3] = 0; };
+    auto fold = [&](const uint32_t(&src)[4]) {
+        x ^= src[0] ^ src[1];
+        x ^= src[2] ^ src[3];
+        s += src[0] + src[1];
+        s += src[2] + src[3];
+    };
+
+    const uint64_t n_batches = (reads + 31) >> 5;
+    uint32_t cur = gen(first + lane);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u * P + sub);
+        if ((uint64_t)(u * P + sub) < reads) issue(line, d[u]); else clear(d[u]);
+    }
+    for (uint64_t b = 0; b < n_batches; ++b) {
+        const uint64_t t0 = b << 5;
+        const uint32_t nxt = gen(first + t0 + 32 + lane);
+        if (t0 + 32 + U * P <= reads) {  // every read of this batch and its refills exist
+#pragma unroll
+            for (int k = 0; k < NL; ++k) {
+                fold(d[k % U]);
+                uint32_t line = (k + U < NL)
+                                    ? __shfl_sync(0xFFFFFFFFu, cur, ((k + U) * P + sub) & 31)
+                                    : __shfl_sync(0xFFFFFFFFu, nxt, ((k + U - NL) * P + sub) & 31);
+                issue(line, d[k % U]);
+            }
+        } else {  // ragged tail: slots that get no read are cleared, so folding them is harmless
+#pragma unroll
+            for (int k = 0; k < NL; ++k) {
+                fold(d[k % U]);
+                uint32_t line = (k + U < NL)
+                                    ? __shfl_sync(0xFFFFFFFFu, cur, ((k + U) * P + sub) & 31)
+                                    : __shfl_sync(0xFFFFFFFFu, nxt, ((k + U - NL) * P + sub) & 31);
+                if (t0 + (uint64_t)((k + U) * P) + sub < reads) issue(line, d[k % U]);
+                else clear(d[k % U]);
+            }
+        }
+        cur = nxt;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        x ^= __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    }
+    X = x;
+    S = s;
+}
+
+template <int W, int U, int VAR>
+__device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
+                                           uint64_t key, uint32_t index_mode, uint64_t v,
+                                           uint64_t V, uint64_t first, uint64_t reads,
+                                           uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
+                                           uint32_t &S, uint32_t *violations)
+{
+    if constexpr (VAR == kVarPacked && W < 4)
+        warp_reads_packed<W, U>(buf, key, index_mode, v, V, first, reads, base, n, lane, X, S);
+    else
+        warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, index_mode, v, V, first,
+                                                   reads, base, n, lane, X, S, violations);
+}
+
+template <int W, int U, int VAR>
 __global__ void __launch_bounds__(1024, 1)
     read_kernel(const __grid_constant__ ReadArgs a, const __grid_constant__ Tables tab)
 {
-    __shared__ uint32_t sh_sm, sh_slot;
+    __shared__ uint32_t sh_sm, sh_slot, sh_workers;
     __shared__ uint16_t sh_group[RR_MAX_SM];
     __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     ScratchHeader *sc = a.scratch;
 
-    if (a.mode == RR_MODE_PER_SM) {
+    if (a.mode == RR_MODE_POOLED) {
+        // Work sharing inside an SM group: items (logical warp, block of reads) come from the
+        // group's counter, so the group's SMs split the group's work however fast each runs.
+        if (threadIdx.x == 0) {
+            uint32_t sm = smid();
+            sh_sm = sm;
+            sh_slot = (sm < a.nsm) ? atomicAdd(&sc->claim[sm], 1u) : 0xFFFFFFFFu;
+            if (sm >= a.nsm) atomicOr(&sc->status, 1u);
+        }
+        for (uint32_t k = threadIdx.x; k < a.nsm; k += blockDim.x) sh_group[k] = tab.group_of_sm[k];
+        for (uint32_t k = threadIdx.x; k < a.n_groups; k += blockDim.x) sh_win[k] = tab.windows[k];
+        __syncthreads();
+        const uint32_t sm = sh_sm, slot = sh_slot;
+        if (slot >= a.cps) return;
+        const uint32_t g = sh_group[sm];
+        if (g == RR_SM_INACTIVE) return;
+        const uint32_t base = sh_win[g].base_line, n = sh_win[g].n_lines;
+        const uint32_t v0 = tab.warp_start[g], cnt = tab.warp_start[g + 1] - v0;
+        // physical warps working for this group: its SMs times the warps of one block
+        if (threadIdx.x == 0) sh_workers = 0;
+        __syncthreads();
+        {
+            uint32_t mine = 0;
+            for (uint32_t k = threadIdx.x; k < a.nsm; k += blockDim.x) mine += sh_group[k] == g;
+            if (mine) atomicAdd(&sh_workers, mine);
+        }
+        __syncthreads();
+        const uint64_t workers = (uint64_t)sh_workers * a.wpc;
+        // The group's work is the line of cnt * reads reads (warp-major).  Grabs shrink as the
+        // line runs out (guided self-scheduling): long runs while there is plenty, so the load
+        // ring is rarely drained, short ones at the end, so no warp is left with a long tail.
+        const uint64_t total = (uint64_t)cnt * a.reads;
+        uint64_t t_start = 0;
+        if (threadIdx.x == 0) t_start = globaltimer();
+        uint32_t *out_words = reinterpret_cast<uint32_t *>(a.out);
+        for (;;) {
+            unsigned long long x = 0, len = 0;
+            if (lane == 0) {
+                const unsigned long long seen =
+                    *reinterpret_cast<volatile unsigned long long *>(&sc->pool_next[g]);
+                const unsigned long long left = total > seen ? total - seen : 0;
+                len = left / (2 * workers);
+                len = min(len, 8192ull) & ~31ull;
+                len = max(len, (unsigned long long)a.pool_block);
+                x = atomicAdd(&sc->pool_next[g], len);
+            }
+            x = __shfl_sync(0xFFFFFFFFu, x, 0);
+            len = __shfl_sync(0xFFFFFFFFu, len, 0);
+            if (x >= total) break;
+            const uint64_t end = (x + len < total) ? (uint64_t)(x + len) : total;
+            while (x < end) {  // a grab may run over the end of one logical warp into the next
+                const uint64_t w = x / a.reads, i0 = x - w * a.reads;
+                const uint64_t n_seg = (end - x < a.reads - i0) ? end - x : a.reads - i0;
+                const uint64_t v = v0 + w;
+                uint32_t X, S;
+                warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode,
+                                          v, a.n_warps, a.first_read + i0, n_seg, base, n, lane, X,
+                                          S, &sc->violations);
+                if (lane == 0) {
+                    atomicXor(&out_words[2 * v], X);
+                    atomicAdd(&out_words[2 * v + 1], S);
+                }
+                x += n_seg;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            BlockRecord r;
+            r.smid = sm;
+            r.slot = slot;
+            r.t_start = t_start;
+            r.t_end = globaltimer();
+            sc->rec[sm * a.cps + slot] = r;
+            atomicAdd(&sc->blocks_run, 1u);
+        }
+    } else if (a.mode == RR_MODE_PER_SM) {
         if (threadIdx.x == 0) {
             uint32_t sm = smid();
             sh_sm = sm;
@@ -153,7 +323,7 @@ __global__ void __launch_bounds__(1024, 1)
         const uint64_t v = (uint64_t)sm * a.wps + slot * a.wpc + warp;
         const uint64_t V = (uint64_t)a.nsm * a.wps;
         uint32_t X, S;
-        warp_reads<W, U, CHECKED>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v, V,
+        warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v, V,
                                   a.first_read, a.reads, base, n, lane, X, S, &sc->violations);
         if (lane == 0) a.out[v] = make_uint2(X, S);
         __syncthreads();
@@ -172,7 +342,7 @@ __global__ void __launch_bounds__(1024, 1)
         const uint64_t stride = (uint64_t)gridDim.x * a.wpc;
         for (uint64_t v = (uint64_t)blockIdx.x * a.wpc + warp; v < a.n_warps; v += stride) {
             uint32_t X, S;
-            warp_reads<W, U, CHECKED>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v,
+            warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v,
                                       a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
                                       &sc->violations);
             if (lane == 0) a.out[v] = make_uint2(X, S);
@@ -223,7 +393,7 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     if (threadIdx.x == 0) t_start = globaltimer();
     const uint64_t v = (uint64_t)sm * a.wps + warp;
     uint32_t X, S;
-    warp_reads<1, kProbeUnroll, false>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
+    warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
                                        RR_INDEX_RANDOM, v, (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
                                        a.n_lines, lane, X, S, nullptr);
     if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
@@ -237,21 +407,34 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
 // ---- host side -------------------------------------------------------------------------------
 typedef void (*ReadKernel)(const ReadArgs, const Tables);
 
-static ReadKernel pick_kernel(uint32_t W, uint32_t U, bool checked)
+static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
 {
-#define RR_ROW(W_)                                                                      \
+    if (variant == RR_VARIANT_PACKED && W < 4) {  // U counts warp loads of 4/W lines each
+#define RR_PACKED_ROW(W_)                                                               \
+    if (W == W_) switch (U) {                                                           \
+            case 1: return read_kernel<W_, 1, kVarPacked>;                              \
+            case 2: return read_kernel<W_, 2, kVarPacked>;                              \
+            case 4: return read_kernel<W_, 4, kVarPacked>;                              \
+            default: return read_kernel<W_, 8, kVarPacked>;                             \
+        }
+        RR_PACKED_ROW(1)
+        RR_PACKED_ROW(2)
+#undef RR_PACKED_ROW
+    }
+    const bool checked = variant == RR_VARIANT_LDG_CHECKED;
+#define RR_ROW(W_, UMAX_)                                                               \
     if (W == W_) {                                                                      \
-        if (checked) return read_kernel<W_, 4, true>;                                   \
+        if (checked) return read_kernel<W_, 4, kVarChecked>;                            \
         switch (U) {                                                                    \
-            case 2: return read_kernel<W_, 2, false>;                                   \
-            case 4: return read_kernel<W_, 4, false>;                                   \
-            case 8: return read_kernel<W_, 8, false>;                                   \
-            case 16: return read_kernel<W_, 16, false>;                                 \
+            case 2: return read_kernel<W_, 2, kVarLdg>;                                 \
+            case 4: return read_kernel<W_, 4, kVarLdg>;                                 \
+            case 8: return read_kernel<W_, 8, kVarLdg>;                                 \
+            case 16: return read_kernel<W_, UMAX_, kVarLdg>;                            \
         }                                                                               \
     }
-    RR_ROW(1)
-    RR_ROW(2)
-    RR_ROW(4)
+    RR_ROW(1, 16)
+    RR_ROW(2, 16)
+    RR_ROW(4, 8)
 #undef RR_ROW
     return nullptr;
 }
@@ -269,11 +452,14 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
                              uint32_t *unroll)
 {
     if (!p || !out || !scratch || !p->buf) return RR_ERR_ARG;
-    if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_PER_SM ||
-        p->index_mode > RR_INDEX_STRIDE || p->variant > RR_VARIANT_LDG_CHECKED || p->reserved)
+    if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_POOLED ||
+        p->index_mode > RR_INDEX_STRIDE || p->variant > RR_VARIANT_PACKED)
         return RR_ERR_ARG;
-    uint32_t U = p->unroll ? p->unroll : 8u;
-    if (U != 2 && U != 4 && U != 8 && U != 16) return RR_ERR_ARG;
+    if (p->mode != RR_MODE_POOLED && (p->pool_block_reads || p->warp_start)) return RR_ERR_ARG;
+    uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_PACKED ? 4u : 8u);
+    if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && p->variant == RR_VARIANT_PACKED))
+        return RR_ERR_ARG;
+    if (U * p->words_per_lane > 32) U = 32 / p->words_per_lane;  // the ring holds 32 words a lane
     *unroll = U;
     if ((uintptr_t)p->buf % 512u) return RR_ERR_ALIGN;
     if ((uintptr_t)out % 8u || (uintptr_t)scratch % 16u) return RR_ERR_ALIGN;
@@ -282,6 +468,27 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     if (p->reads_per_warp > (1ull << 62) || p->first_read > (1ull << 62)) return RR_ERR_RANGE;
     if (p->mode == RR_MODE_LOGICAL) {
         if (p->n_warps == 0 || p->group_of_sm || p->windows || p->n_groups) return RR_ERR_ARG;
+    } else if (p->mode == RR_MODE_POOLED) {
+        const uint32_t w = p->warps_per_sm;
+        if (w == 0 || w > RR_MAX_WARPS_PER_SM || p->nsm == 0 || p->nsm > RR_MAX_SM) return RR_ERR_ARG;
+        if (!p->group_of_sm || !p->windows || !p->warp_start || p->n_groups == 0 ||
+            p->n_groups > RR_MAX_GROUPS || p->n_warps == 0 || p->index_mode != RR_INDEX_RANDOM ||
+            p->pool_block_reads > (1u << 20))
+            return RR_ERR_ARG;
+        if (p->warp_start[0] != 0 || p->warp_start[p->n_groups] != p->n_warps) return RR_ERR_ARG;
+        std::vector<bool> served(p->n_groups, false);
+        for (uint32_t s = 0; s < p->nsm; ++s) {
+            if (p->group_of_sm[s] == RR_SM_INACTIVE) continue;
+            if (p->group_of_sm[s] >= p->n_groups) return RR_ERR_MAP;
+            served[p->group_of_sm[s]] = true;
+        }
+        for (uint32_t g = 0; g < p->n_groups; ++g) {
+            if (p->warp_start[g + 1] < p->warp_start[g]) return RR_ERR_ARG;
+            if (p->windows[g].n_lines == 0 ||
+                (uint64_t)p->windows[g].base_line + p->windows[g].n_lines > L)
+                return RR_ERR_RANGE;
+            if (p->warp_start[g + 1] > p->warp_start[g] && !served[g]) return RR_ERR_MAP;
+        }
     } else {
         const uint32_t w = p->warps_per_sm;
         if (w == 0 || w > RR_MAX_WARPS_PER_SM) return RR_ERR_ARG;
@@ -309,7 +516,7 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
 
 static int32_t geometry(const rr_read_params_t *p, const DeviceFacts &f, Geometry *g)
 {
-    if (p->mode == RR_MODE_PER_SM) {
+    if (p->mode != RR_MODE_LOGICAL) {
         if (p->nsm && p->nsm != (uint32_t)f.nsm) return RR_ERR_ARG;
         g->wps = p->warps_per_sm;
         g->cps = g->wps > 32 ? 2 : 1;
@@ -318,7 +525,7 @@ static int32_t geometry(const rr_read_params_t *p, const DeviceFacts &f, Geometr
         g->active_sms = 0;
         for (int s = 0; s < f.nsm; ++s)
             g->active_sms += !p->group_of_sm || p->group_of_sm[s] != RR_SM_INACTIVE;
-        g->active_warps = g->active_sms * g->wps;
+        g->active_warps = p->mode == RR_MODE_POOLED ? p->n_warps : g->active_sms * g->wps;
     } else {
         g->wps = g->wpc = 32;
         g->cps = 1;
@@ -376,7 +583,7 @@ static int32_t decode(const rr_read_params_t *p, const Geometry &g, const Device
         t1 = std::max(t1, r.t_end);
         return true;
     };
-    if (p->mode == RR_MODE_PER_SM) {
+    if (p->mode != RR_MODE_LOGICAL) {
         for (int s = 0; s < f.nsm; ++s) {
             if (p->group_of_sm && p->group_of_sm[s] == RR_SM_INACTIVE) continue;
             bool all = true;
@@ -418,13 +625,12 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     Geometry g;
     rc = geometry(p, f, &g);
     if (rc != RR_OK) return rc;
-    const bool checked = p->variant == RR_VARIANT_LDG_CHECKED;
-    ReadKernel kernel = pick_kernel(p->words_per_lane, U, checked);
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant);
     if (!kernel) return RR_ERR_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
 
     size_t smem = 0;
-    if (p->mode == RR_MODE_PER_SM) {
+    if (p->mode != RR_MODE_LOGICAL) {
         rc = ballast_for_occupancy(kernel, (int)g.block, (int)g.cps, f, &smem);
         if (rc != RR_OK) return rc;
     }
@@ -444,6 +650,7 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     a.cps = g.cps;
     a.nsm = (uint32_t)f.nsm;
     a.n_groups = p->group_of_sm ? p->n_groups : 0;
+    a.pool_block = p->pool_block_reads ? p->pool_block_reads : 64u;
     a.out = (uint2 *)out_dev;
     a.scratch = (ScratchHeader *)scratch_dev;
     Tables tab;
@@ -452,6 +659,8 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
         std::memcpy(tab.group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
         std::memcpy(tab.windows, p->windows, sizeof(rr_window_t) * p->n_groups);
     }
+    if (p->mode == RR_MODE_POOLED)
+        std::memcpy(tab.warp_start, p->warp_start, sizeof(uint32_t) * (p->n_groups + 1));
 
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (res) {
@@ -476,6 +685,11 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     RR_CUDA_C(cudaMemsetAsync(scratch_dev, 0, offsetof(ScratchHeader, probe), stream));
     if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
         RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
+    if (p->mode == RR_MODE_POOLED) {  // work counters, and the checksums the atomics add into
+        RR_CUDA_C(cudaMemsetAsync(&((ScratchHeader *)scratch_dev)->pool_next, 0,
+                                  sizeof(unsigned long long) * RR_MAX_GROUPS, stream));
+        RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)p->n_warps * sizeof(uint2), stream));
+    }
     if (res) RR_CUDA_C(cudaEventRecord(e0, stream));
     kernel<<<g.grid, g.block, smem, stream>>>(a, tab);
     RR_CUDA_C(cudaGetLastError());
@@ -512,6 +726,23 @@ extern "C" int32_t rr_read_report(const rr_read_params_t *p, const void *scratch
                             cudaMemcpyDeviceToHost, stream));
     RR_CUDA(cudaStreamSynchronize(stream));
     return decode(p, g, f, h, 0.0, res);
+}
+
+extern "C" int32_t rr_read_block_times(const void *scratch_dev, uint32_t nsm, uint64_t *t_start,
+                                       uint64_t *t_end, void *stream_)
+{
+    if (!scratch_dev || !t_start || !t_end || nsm == 0 || nsm > RR_MAX_SM) return RR_ERR_ARG;
+    if ((uintptr_t)scratch_dev % 16u) return RR_ERR_ALIGN;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    static thread_local ScratchHeader h;
+    RR_CUDA(cudaMemcpyAsync(&h, scratch_dev, offsetof(ScratchHeader, probe),
+                            cudaMemcpyDeviceToHost, stream));
+    RR_CUDA(cudaStreamSynchronize(stream));
+    for (uint32_t s = 0; s < nsm; ++s) {  // one block per SM: record index = SM id
+        t_start[s] = h.rec[s].t_end ? h.rec[s].t_start : 0;
+        t_end[s] = h.rec[s].t_end;
+    }
+    return RR_OK;
 }
 
 // ---- probes ------------------------------------------------------------------------------------
@@ -755,6 +986,7 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     // validate against a stand-in scratch address first: argument errors come before any CUDA call
     int32_t rc = validate_read(p, out_dev, (const void *)256, &U);
     if (rc != RR_OK) return rc;
+    if (p->mode == RR_MODE_POOLED) return RR_ERR_STATIC_LIMIT;
     if (p->mode == RR_MODE_PER_SM && (p->warps_per_sm > 32 || p->nsm > kStaticMaxSm))
         return RR_ERR_STATIC_LIMIT;
     DeviceFacts f;
@@ -765,7 +997,7 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     rc = geometry(p, f, &g);
     if (rc != RR_OK) return rc;
     if (g.cps != 1 || g.grid > kStaticMaxSm) return RR_ERR_STATIC_LIMIT;
-    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant == RR_VARIANT_LDG_CHECKED);
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant);
     if (!kernel) return RR_ERR_ARG;
     void *scratch = nullptr;
     rc = static_scratch_address(f.device, &scratch);
@@ -791,6 +1023,7 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     a.cps = g.cps;
     a.nsm = (uint32_t)f.nsm;
     a.n_groups = p->group_of_sm ? p->n_groups : 0;
+    a.pool_block = 256u;
     a.out = (uint2 *)out_dev;
     a.scratch = (ScratchHeader *)scratch;
     Tables tab;

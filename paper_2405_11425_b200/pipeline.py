@@ -169,6 +169,94 @@ class Session:
         return rr.rr_make_windows(region_bytes or self.region_bytes, W, window_bytes,
                                   groups.n_groups)
 
+    # -- Section 2.3: every group on its own; work in proportion to capacity ---------------------
+    def measure_group_rates(self, groups: Groups, window_bytes: int, *, W: int = 1,
+                            reads_per_warp: int = 256 * 8, seed: int = 23) -> list:
+        """GB/s of each group running alone inside one window of `window_bytes` (below the reach)."""
+        n_lines = max(1, min(window_bytes, self.region_bytes) // (128 * W))
+        rates = []
+        for g in range(groups.n_groups):
+            only = np.where(groups.group_of_sm == g, 0, rr.RR_SM_INACTIVE).astype(np.uint16)
+            rate, _ = self.read(self.region_bytes, W=W, seed=seed, reads_per_warp=reads_per_warp,
+                                group_of_sm=only, windows=[[0, n_lines]], reps=3, warm=1)
+            rates.append(rate)
+        return rates
+
+    def balanced_plan(self, groups: Groups, rates, n_warps: int, *, W: int = 1,
+                      max_window_bytes: int = 0, region_bytes=None):
+        """Windows and logical-warp ranges in proportion to the groups' measured rates
+        (weights = rates in MB/s).  Returns (windows, warp_start)."""
+        weights = np.maximum(1, np.rint(np.asarray(rates, dtype=np.float64) * 1000.0)).astype(
+            np.uint32)
+        return rr.rr_make_weighted_windows(region_bytes or self.region_bytes, W, weights, n_warps,
+                                           max_window_bytes)
+
+    def balance(self, groups: Groups, *, W: int = 1, n_warps: int | None = None,
+                reads_per_warp: int = 256 * 64, seed: int = 23, max_window_bytes: int = 0,
+                rounds: int = 6, spread_goal: float = 0.02, start_rates=None,
+                launches_per_round: int = 1, **kw):
+        """Closed-loop version of balanced_plan: run the pooled workload, see from the per-SM
+        timers when each group finished, move work (and window size) towards the groups that
+        finished early, repeat.  Needed because a group's capacity with every other group
+        running differs from its capacity alone.  Stops after `rounds` rounds or once the
+        groups' finish times lie within `spread_goal` of each other.  Each round queues
+        `launches_per_round` launches back to back and reads the timers of the last one: under
+        sustained load the clocks settle lower than in a single burst, and the groups whose
+        limit follows the clock lose capacity while the others do not.  Returns (windows,
+        warp_start, weights, [GB/s of each round, from the device timers])."""
+        n_warps = n_warps or self.nsm * 32
+        G = groups.n_groups
+        if start_rates is None:
+            weights = np.full(G, 1000, dtype=np.uint32)
+        else:
+            weights = np.maximum(1, np.rint(np.asarray(start_rates, np.float64) * 1000)).astype(
+                np.uint32)
+        history = []
+        for _ in range(rounds):
+            win, ws = rr.rr_make_weighted_windows(self.region_bytes, W, weights, n_warps,
+                                                  max_window_bytes)
+            p = self.params(None, mode=rr.RR_MODE_POOLED, n_warps=n_warps, W=W,
+                            reads_per_warp=reads_per_warp, seed=seed,
+                            group_of_sm=groups.group_of_sm, windows=win, warp_start=ws, **kw)
+            for _ in range(max(1, launches_per_round)):
+                rr.rr_random_read(p, self.out, self.scratch, timed=False)
+            t0, t1 = rr.rr_read_block_times(self.scratch, self.nsm)
+            ran = t1 > 0
+            begin = t0[ran].min()
+            history.append(n_warps * reads_per_warp * 128 * W / float(t1[ran].max() - begin))
+            work = np.diff(ws.astype(np.int64)).astype(np.float64)
+            rate = np.zeros(G)
+            finish = np.zeros(G)
+            for g in range(G):
+                m = (groups.group_of_sm == g) & ran
+                finish[g] = max(1.0, float(t1[m].max() - begin)) if m.any() else 0.0
+                rate[g] = work[g] / finish[g] if m.any() else 0.0
+            seen = finish[finish > 0]
+            if (seen.max() - seen.min()) / seen.max() <= spread_goal:
+                break
+            rate = np.maximum(rate, rate[rate > 0].min() * 1e-3)
+            weights = np.maximum(1, np.rint(rate / rate.sum() * 1e6)).astype(np.uint32)
+        win, ws = rr.rr_make_weighted_windows(self.region_bytes, W, weights, n_warps,
+                                              max_window_bytes)
+        return win, ws, weights, history
+
+    def read_pooled(self, groups: Groups, windows, warp_start, *, region_bytes=None,
+                    reps: int = 3, warm: int = 1, out=None, **kw):
+        """Median GB/s of pooled-mode launches; `out` must hold warp_start[-1] checksum pairs."""
+        n_warps = int(warp_start[-1])
+        if out is None:
+            out = self.out
+        if out.shape[0] < n_warps:
+            raise ValueError("output buffer smaller than the number of logical warps")
+        p = self.params(region_bytes, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
+                        group_of_sm=groups.group_of_sm, windows=windows, warp_start=warp_start,
+                        **kw)
+        for _ in range(warm):
+            rr.rr_random_read(p, out, self.scratch)
+        res = [rr.rr_random_read(p, out, self.scratch) for _ in range(reps)]
+        rates = sorted(r.gbps for r in res)
+        return rates[(len(rates) - 1) // 2], res[-1]
+
     def naive_control(self, window_bytes: int, seed: int, W: int = 1, region_bytes=None):
         """The paper's per-SM control: every SM on its own picks a pseudo-random chunk."""
         win, cov = rr.rr_make_windows(region_bytes or self.region_bytes, W, window_bytes, self.nsm,

@@ -129,6 +129,52 @@ def test_make_windows_matches_oracle():
         rr.rr_make_windows(64, 1, 1 << 10, 2)
 
 
+def test_weighted_windows_match_oracle():
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        G = int(rng.integers(1, 40))
+        w = rng.integers(1, 5000, G).astype(np.uint32)
+        W = int(rng.choice([1, 2, 4]))
+        region = int(rng.integers(G * 2000, 10 ** 8)) * 128 * W + 9
+        V = int(rng.integers(G * 50, 10 ** 5))
+        try:
+            b_win, b_ws = oracle.make_weighted_windows(region, W, w, V)
+        except oracle.OracleError:                   # a tiny weight left a group without warps
+            with pytest.raises(rr.RRError):
+                rr.rr_make_weighted_windows(region, W, w, V)
+            continue
+        a_win, a_ws = rr.rr_make_weighted_windows(region, W, w, V)
+        assert np.array_equal(a_win, b_win) and np.array_equal(a_ws, b_ws)
+    big = int(0.95 * 178 * (1 << 30)) // 512 * 512
+    w = [249, 249, 250, 251, 138, 248] * 4
+    a = rr.rr_make_weighted_windows(big, 1, w, 4736, max_window_bytes=70 << 30)
+    b = oracle.make_weighted_windows(big, 1, w, 4736, max_window_bytes=70 << 30)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    for bad in (dict(weights=[1, 0, 1], n_warps=100), dict(weights=[1, 1, 1], n_warps=2),
+                dict(weights=[2 ** 31, 2 ** 31], n_warps=100)):
+        with pytest.raises(rr.RRError):
+            rr.rr_make_weighted_windows(1 << 30, 1, bad["weights"], bad["n_warps"])
+    with pytest.raises(rr.RRError):
+        rr.rr_make_weighted_windows(1 << 30, 1, [1, 3], 100, max_window_bytes=600 << 20)
+
+
+def test_pooled_mode_argument_errors():
+    g = np.array([0, 1, 0, 1], np.uint16)
+    ok = dict(mode=rr.RR_MODE_POOLED, n_warps=10, nsm=4, warps_per_sm=8, group_of_sm=g,
+              windows=[[0, 100], [100, 100]], warp_start=[0, 4, 10])
+    assert _call(**{**ok, "warp_start": None}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "warp_start": [1, 4, 10]}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "warp_start": [0, 4, 9]}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "warp_start": [0, 11, 10]}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "index_mode": rr.RR_INDEX_STRIDE}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "windows": [[0, 100], [100, 90000]]}) == rr.RR_ERR_RANGE
+    assert _call(**{**ok, "group_of_sm": np.array([0, 0, 0, 0], np.uint16)}) == rr.RR_ERR_MAP
+    assert _call(**{**ok, "group_of_sm": np.array([0, 2, 0, 1], np.uint16)}) == rr.RR_ERR_MAP
+    # other modes take no pool arguments
+    assert _call(pool_block_reads=256) == rr.RR_ERR_ARG
+    assert _call(warp_start=[0, 4]) == rr.RR_ERR_ARG
+
+
 def test_reach_matches_oracle():
     rng = np.random.default_rng(3)
     sizes = [s << 30 for s in (1, 4, 16, 32, 48, 64, 96, 128, 160, 169)]

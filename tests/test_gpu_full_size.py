@@ -163,3 +163,29 @@ def test_contention_groups_nest_inside_gpcs(ses):
         assert len(set(gpc[members].tolist())) <= 1, (k, np.where(groups.group_of_sm == k)[0])
     # and the partition is finer than the GPCs, as the paper found on its card
     assert groups.n_groups > int((np.bincount(gpc) > 2).sum())
+
+
+def test_pooled_bench_launch_configuration_sampled(ses):
+    # the launch bench.py times: 148 x 32 logical warps owned by 24 SM groups in proportion to
+    # their weights, windows tiling the whole buffer, 16384 reads per warp
+    region = ses.region_bytes
+    groups = rr_inputs.synthetic_group_map(ses.nsm, 24, seed=7)
+    weights = [30000 if g % 8 == 0 else 43000 + 100 * g for g in range(24)]
+    n_warps = ses.nsm * WPS
+    win, ws = rr.rr_make_weighted_windows(region, 1, weights, n_warps, max_window_bytes=64 * GiB)
+    assert int(win[-1, 0]) + int(win[-1, 1]) == region // 128 and ws[-1] == n_warps
+    reads, first = 256 * 64, 256 * 64 * 5
+    p = ses.params(region, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps, warps_per_sm=WPS,
+                   reads_per_warp=reads, first_read=first, seed=rr_inputs.CFG4_SEED,
+                   group_of_sm=groups, windows=win, warp_start=ws)
+    assert rr.rr_random_read(p, ses.out, ses.scratch, timed=False) is None
+    rep = rr.rr_read_report(p, ses.scratch)
+    assert rep.sms_covered == ses.nsm and rep.bytes == n_warps * reads * 128
+    got = ses.checksums(n_warps)
+    for v in _sample(n_warps):
+        g = int(np.searchsorted(ws, v, side="right") - 1)
+        base, n = map(int, win[g])
+        assert tuple(got[v]) == oracle.warp_checksum(rr_inputs.CFG4_SEED, v, first, reads, 1, base,
+                                                     n), v
+    t0, t1 = rr.rr_read_block_times(ses.scratch, ses.nsm)
+    assert (t1 > t0).all() and t0.min() > 0

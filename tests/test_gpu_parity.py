@@ -260,3 +260,91 @@ def test_gpc_map_from_cluster_placement(dev):
     assert n2 == n_gpcs and np.array_equal(g, g2)      # placement facts, not timing: repeatable
     with pytest.raises(rr.RRError):
         rr.rr_gpc_map(dev.scratch, dev.nsm + 1)
+
+
+@pytest.mark.parametrize("W,block", [(1, 0), (1, 64), (2, 100), (4, 1000)])
+def test_pooled_mode_matches_oracle(dev, W, block):
+    region = 900 * MiB + 128
+    G = 7
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=9, inactive_frac=0.1)
+    weights = [5, 1, 3, 3, 2, 8, 4]
+    n_warps = 1500
+    win, ws = rr.rr_make_weighted_windows(region, W, weights, n_warps)
+    reads, first = 333, 17                       # not a multiple of the block: ragged last item
+    out = _out(dev, n_warps)                     # poisoned: the call must clear it
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
+                      warps_per_sm=16, nsm=dev.nsm, reads_per_warp=reads, first_read=first, seed=23,
+                      group_of_sm=groups, windows=win, warp_start=ws, pool_block_reads=block)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    expect = oracle.read_pooled(region, W, win, ws, reads, 23, first_read=first)
+    assert np.array_equal(_np(out), expect)
+    assert res.bytes == n_warps * reads * 128 * W
+    assert res.sms_covered == int((groups != 0xFFFF).sum())
+    # twice in a row: counters and outputs are cleared by the call
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), expect)
+
+
+def test_pooled_mode_empty_group_and_zero_reads(dev):
+    region = 64 * MiB
+    groups = np.zeros(dev.nsm, np.uint16)
+    groups[1::2] = 2                                # group 1 owns no warps and has no SM
+    win = np.array([[0, 1000], [1000, 1000], [5000, 777]], np.uint32)
+    ws = [0, 40, 40, 100]
+    out = _out(dev, 100)
+    p = rr.ReadParams(dev.buf, region, mode=rr.RR_MODE_POOLED, n_warps=100, warps_per_sm=4,
+                      nsm=dev.nsm, reads_per_warp=50, seed=3, group_of_sm=groups, windows=win,
+                      warp_start=ws)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_pooled(region, 1, win, ws, 50, 3))
+    p0 = rr.ReadParams(dev.buf, region, mode=rr.RR_MODE_POOLED, n_warps=100, warps_per_sm=4,
+                       nsm=dev.nsm, reads_per_warp=0, seed=3, group_of_sm=groups, windows=win,
+                       warp_start=ws)
+    rr.rr_random_read(p0, out, dev.scratch)
+    assert not _np(out).any()
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+@pytest.mark.parametrize("unroll", [0, 2, 4, 8, 16])
+def test_packed_variant_logical_ragged_reads(dev, W, unroll):
+    region = 777 * MiB + 384
+    for reads, first in [(0, 0), (1, 0), (2, 5), (3, 0), (7, 3), (31, 0), (32, 1), (33, 0),
+                         (40, 100), (61, 7), (64, 0), (100, 9), (257, 2)]:
+        n_warps = 200
+        out = _out(dev, n_warps)
+        p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
+                          reads_per_warp=reads, first_read=first, seed=11, unroll=unroll,
+                          variant=rr.RR_VARIANT_PACKED)
+        rr.rr_random_read(p, out, dev.scratch)
+        expect = oracle.read_logical(region, W, n_warps, reads, 11, first_read=first)
+        assert np.array_equal(_np(out), expect), (W, unroll, reads, first)
+
+
+@pytest.mark.parametrize("W", [1, 2])
+def test_packed_variant_grouped_pooled_and_stride(dev, W):
+    region = dev.buf_bytes
+    G = 6
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=2, inactive_frac=0.05)
+    windows, _ = rr.rr_make_windows(region, W, region // 4, G)
+    windows[2] = (123, 1001)
+    out = _out(dev, dev.nsm * 32)
+    p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=32, reads_per_warp=133, seed=23,
+                      group_of_sm=groups, windows=windows, variant=rr.RR_VARIANT_PACKED)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_per_sm(region, W, dev.nsm, 32, 133, 23,
+                                                       group_of_sm=groups, windows=windows))
+    win, ws = rr.rr_make_weighted_windows(region, W, [3, 1, 2, 2, 5, 1], 999)
+    out = _out(dev, 999)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_POOLED, n_warps=999, warps_per_sm=32,
+                      nsm=dev.nsm, reads_per_warp=301, seed=5, group_of_sm=groups, windows=win,
+                      warp_start=ws, variant=rr.RR_VARIANT_PACKED)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_pooled(region, W, win, ws, 301, 5))
+    V, R = 64, 96
+    small = V * R * 128 * W
+    out = _out(dev, V)
+    p = rr.ReadParams(dev.buf, small, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=V, reads_per_warp=R,
+                      index_mode=rr.RR_INDEX_STRIDE, variant=rr.RR_VARIANT_PACKED)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_logical(small, W, V, R, 0,
+                                                        index_mode=oracle.INDEX_STRIDE))
