@@ -388,7 +388,7 @@ def run_gpu(args):
 
 # DRAM bytes moved per algorithmic byte by the read kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over lines x 128 B, 4 GiB case).
-TRAFFIC_PER_ALGORITHMIC_BYTE = 0.981
+TRAFFIC_PER_ALGORITHMIC_BYTE = 0.975
 
 
 def main():
