@@ -149,6 +149,40 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                                                            reads_per_warp=reads),
                                "windows": rows}
     R["cfg4_grouped"] = cfg4
+
+    # work in proportion to group capacity (pooled mode), balanced under sustained load
+    balanced = {}
+    n_warps = ses.nsm * 32
+    max_window = reach.reach_bytes if reach.cliff else 0
+    for W, variant, unroll, name in ((1, rr.RR_VARIANT_PACKED, 2, "128B packed"),
+                                     (1, rr.RR_VARIANT_LDG, 8, "128B 32-lane"),
+                                     (2, rr.RR_VARIANT_LDG, 8, "256B 32-lane")):
+        win, ws, weights, hist = ses.balance(groups, W=W, n_warps=n_warps, reads_per_warp=reads,
+                                             seed=23, max_window_bytes=max_window,
+                                             launches_per_round=20 if quick else 150,
+                                             variant=variant, unroll=unroll)
+        p = ses.params(N, W=W, mode=rr.RR_MODE_POOLED, n_warps=n_warps, reads_per_warp=reads,
+                       seed=23, group_of_sm=groups.group_of_sm, windows=win, warp_start=ws,
+                       variant=variant, unroll=unroll)
+        torch.cuda.synchronize()
+        time.sleep(1.0)
+        burst = rr.rr_random_read(p, ses.out, ses.scratch).gbps      # first launch after a pause
+        n = 50 if quick else 500
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(20 if quick else 150):
+            rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+        e0.record()
+        for _ in range(n):
+            rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+        e1.record()
+        torch.cuda.synchronize()
+        rep = rr.rr_read_report(p, ses.scratch)
+        balanced[name] = {"burst_gbps": burst,
+                          "sustained_gbps": rep.bytes * n / e0.elapsed_time(e1) * 1e-6,
+                          "gbps_by_balancing_round": hist, "weights": weights.tolist(),
+                          "window_gib_min_max": [float(win[:, 1].min()) * 128 * W / GiB,
+                                                 float(win[:, 1].max()) * 128 * W / GiB]}
+    R["balanced_pooled"] = balanced
     R["seconds"] = time.time() - t_start
     (out_dir / "report.json").write_text(json.dumps(R, indent=1))
     (out_dir / "report.md").write_text(markdown(R))
@@ -208,6 +242,12 @@ def markdown(R: dict) -> str:
             L.append(f"| {name} | {r['window_gib']:.1f} | {r['coverage']:.2f} | {f(r['grouped'])} | "
                      f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} |")
         L.append("")
+    L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
+          "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]
+    for name, b in R.get("balanced_pooled", {}).items():
+        L.append(f"| {name} | {b['burst_gbps']:.0f} | {b['sustained_gbps']:.0f} | "
+                 f"{b['window_gib_min_max'][0]:.1f}-{b['window_gib_min_max'][1]:.1f} |")
+    L.append("")
     L.append(f"total {R['seconds']:.0f} s")
     return "\n".join(L) + "\n"
 
