@@ -250,7 +250,8 @@ int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint6
  * Paper, Section 2.2 and Figure 3 ("rearranging the indices" so groups show as blocks).  Here:
  * symmetrise, quantise against the median, average-linkage agglomeration with exact integer
  * sums, cut at the largest height gap among cuts leaving 2..n/3 clusters, null rule (gap below
- * 4 robust standard deviations of the height -> one group), groups numbered by their smallest
+ * 4 robust standard deviations of the height, or below 1 % of the median pair rate -- the paper
+ * sets the faint background pattern aside -- gives one group), groups numbered by their smallest
  * SM id.  Runs as one block on the device.
  * T_host: HOST n*n float32 row-major; off-diagonal entries must be finite and > 0, else
  * RR_ERR_ARG; 2 <= n <= RR_MAX_SM.  flags = 0: the diagonal is ignored.

@@ -300,7 +300,8 @@ int32_t orc_read_pooled(uint64_t region_bytes, uint32_t W, uint32_t n_groups,
  *    clusters to maximise h[k] - h[k-1]; the first maximum wins
  * 5. null rule: sigma = 1.4826 * MAD of the q of pairs in different clusters after
  *    the cut, divided by sqrt of the number of pairs averaged in merge k (so it
- *    is the noise of the height that defines the gap); gap < 4 sigma -> one group
+ *    is the noise of the height that defines the gap); gap < 4 sigma, or gap below
+ *    1 % of the median pair rate (a faint background pattern) -> one group
  * 6. labels: groups numbered by their smallest SM id
  * heights (optional) receives the n-1 merge heights.                            */
 static int cmp_double(const void *a, const void *b)
@@ -455,7 +456,9 @@ int32_t orc_cluster(const float *T, uint32_t n, uint32_t flags, int32_t *group_o
         double sigma = (1.4826 * mad) / sqrt((double)merge_pairs[best_k]);
         double conf = sigma > 0.0 ? best_gap / sigma : (best_gap > 0.0 ? INFINITY : 0.0);
         if (confidence) *confidence = conf;
-        if (!(best_gap >= 4.0 * sigma) || !(best_gap > 0.0)) goto done; /* one group */
+        /* the paper sets the "more faint pattern in the background" aside (Section 2.2):
+         * a gap below 1 % of the median pair rate (2^20 in these units) is no group boundary */
+        if (!(best_gap >= 4.0 * sigma) || !(best_gap >= 10485.76)) goto done; /* one group */
         /* 6. canonical labels: representatives are smallest members */
         uint32_t G = 0;
         for (uint32_t i = 0; i < n; ++i)

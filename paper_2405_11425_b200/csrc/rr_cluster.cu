@@ -268,7 +268,8 @@ __global__ void __launch_bounds__(kClusterThreads, 1) cluster_kernel(uint8_t *wo
         const double gap = out->gap;
         const double conf = sigma > 0.0 ? __ddiv_rn(gap, sigma) : (gap > 0.0 ? INFINITY : 0.0);
         out->confidence = conf;
-        if (gap >= __dmul_rn(4.0, sigma) && gap > 0.0) {
+        // a gap below 1 % of the median pair rate (2^20 in these units) is background, not a group
+        if (gap >= __dmul_rn(4.0, sigma) && gap >= 10485.76) {
             // 6. groups numbered by their smallest SM id (a cluster is named by its smallest member)
             uint32_t G = 0;
             for (uint32_t i = 0; i < n; ++i)

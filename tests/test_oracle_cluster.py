@@ -143,3 +143,21 @@ def test_solo_normalisation_is_scale_free_and_checks_the_diagonal():
     with pytest.raises(oracle.OracleError):
         oracle.cluster(B, solo_normalise=True)
     oracle.cluster(B)      # without the flag the diagonal is ignored
+
+
+def test_faint_background_pattern_is_not_a_grouping():
+    # an almost flat matrix (0.02 % structure, as measured inside the reach on B200) must give one
+    # group however small its noise is: the paper ignores the faint pattern behind the boxes
+    rng = np.random.default_rng(0)
+    n = 148
+    T = np.full((n, n), 150.0) * (1 + 2e-5 * rng.standard_normal((n, n)))
+    T[:4, :] *= 0.9998
+    T[:, :4] *= 0.9998
+    np.fill_diagonal(T, 75.0)
+    g, G, conf, _ = oracle.cluster(T.astype(np.float32), solo_normalise=True)
+    assert G == 1 and not g.any()
+    # a 3 % same-group drop with equally small noise is a grouping
+    T2, truth = rr_inputs.planted_matrix([6] * 12 + [8] * 4, 0.03, seed=1, tpc_drop=0.0,
+                                         background=0.0, sigma=2e-5)
+    g, G, conf, _ = oracle.cluster(T2, solo_normalise=True)
+    assert G == 16 and np.array_equal(g, truth)
