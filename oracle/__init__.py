@@ -63,6 +63,8 @@ def _load():
         lib.orc_warp_checksum.argtypes = [u32, u64, u64, u64, u64, u64, u32, u64, u64, p, p]
         lib.orc_read_logical.restype = i32
         lib.orc_read_logical.argtypes = [u64, u32, u32, u64, u64, u64, u64, p]
+        lib.orc_read_logical_materialised.restype = i32
+        lib.orc_read_logical_materialised.argtypes = [p, u64, u32, u64, u64, u64, u64, p]
         lib.orc_read_per_sm.restype = i32
         lib.orc_read_per_sm.argtypes = [u64, u32, u32, u32, u32, u64, u64, u64, p, p, p, u32, p]
         lib.orc_make_windows.restype = i32
@@ -131,6 +133,18 @@ def read_logical(region_bytes: int, W: int, n_warps: int, reads: int, seed: int,
     out = np.zeros((n_warps, 2), dtype=np.uint32)
     rc = _load().orc_read_logical(region_bytes, W, index_mode, n_warps, first_read, reads, seed,
                                   _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def read_logical_materialised(buf: np.ndarray, W: int, n_warps: int, reads: int, seed: int,
+                              first_read: int = 0) -> np.ndarray:
+    """Logical-mode checksums read from a real host buffer (uint32 words, see fill())."""
+    buf = np.ascontiguousarray(buf, dtype=np.uint32)
+    out = np.zeros((n_warps, 2), dtype=np.uint32)
+    rc = _load().orc_read_logical_materialised(_ptr(buf), buf.size * 4, W, n_warps, first_read,
+                                               reads, seed, _ptr(out))
     if rc != 0:
         raise OracleError(rc)
     return out

@@ -18,8 +18,8 @@
  *     here: average-linkage agglomeration with a largest-gap cut.
  *
  * Everything is written as the definition, one word at a time, with no blocking,
- * fusion or reordering.  The only parallelism is an OpenMP loop over warps, which
- * are independent by definition.
+ * fusion or reordering.  The only parallelism is an OpenMP loop over warps (or over
+ * the words of a fill), which are independent by definition.
  *
  * Pins (see tests/test_oracle_*.py): the public SplitMix64 output streams, a
  * big-integer brute force over tiny materialised buffers, window invariants,
@@ -64,8 +64,10 @@ uint32_t orc_word(uint64_t i)
 
 void orc_fill(uint32_t *dst, uint64_t first_word, uint64_t n_words)
 {
-    for (uint64_t k = 0; k < n_words; ++k)
-        dst[k] = orc_word(first_word + k);
+    int64_t n = (int64_t)n_words;
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < n; ++k)
+        dst[k] = orc_word(first_word + (uint64_t)k);
 }
 
 /* ---- O2: line index ----------------------------------------------------------
@@ -122,6 +124,35 @@ void orc_warp_checksum(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t 
 }
 
 static int orc_width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
+
+/* The same logical-mode read performed on a real buffer in host memory (filled with
+ * orc_fill): the line is indexed literally instead of regenerated.  This is the CPU
+ * analogue of the method for sizes that fit host RAM, and a second statement of what a
+ * "coalesced line read" touches.  buf holds region_bytes/4 words.                     */
+int32_t orc_read_logical_materialised(const uint32_t *buf, uint64_t region_bytes, uint32_t W,
+                                      uint64_t n_warps, uint64_t first_read, uint64_t reads,
+                                      uint64_t seed, uint32_t *out)
+{
+    if (!buf || !out || !orc_width_ok(W)) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    int64_t nw = (int64_t)n_warps;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t x = 0, s = 0;
+        for (uint64_t t = 0; t < reads; ++t) {
+            uint64_t line = orc_draw(seed, (uint64_t)v, first_read + t) % L;
+            const uint32_t *p = buf + line * 32u * W; /* the 32*W words of that line */
+            for (uint32_t k = 0; k < 32u * W; ++k) {
+                x ^= p[k];
+                s += p[k];
+            }
+        }
+        out[2 * v] = x;
+        out[2 * v + 1] = s;
+    }
+    return ORC_OK;
+}
 
 /* Logical-warp mode: v = 0 .. n_warps-1, window = the whole region.
  * out holds n_warps pairs {X, S}.                                               */

@@ -57,6 +57,27 @@ def aggregate_throughput(local_bytes: float, local_seconds: float, group=None) -
     return float(b.item()), float(s.item())
 
 
+def rebalanced_weights(work, finish_ns, scale: int = 1_000_000) -> np.ndarray:
+    """New integer group weights from one balanced-run observation: a group that did `work`
+    units and finished after `finish_ns` has shown a rate work/finish; weights are those rates,
+    normalised to sum to about `scale`.  Groups that were not seen (finish 0) keep a token weight
+    of one thousandth of the slowest observed rate."""
+    work = np.asarray(work, dtype=np.float64)
+    finish = np.asarray(finish_ns, dtype=np.float64)
+    rate = np.where(finish > 0, work / np.maximum(finish, 1.0), 0.0)
+    if not (rate > 0).any():
+        raise ValueError("no group finished any work")
+    rate = np.maximum(rate, rate[rate > 0].min() * 1e-3)
+    return np.maximum(1, np.rint(rate / rate.sum() * scale)).astype(np.uint32)
+
+
+def finish_spread(finish_ns) -> float:
+    """(latest - earliest) / latest over the groups that ran."""
+    f = np.asarray(finish_ns, dtype=np.float64)
+    f = f[f > 0]
+    return float((f.max() - f.min()) / f.max()) if f.size else 0.0
+
+
 class Session:
     """Device buffers of one GPU plus the calls of the path."""
 
@@ -225,17 +246,13 @@ class Session:
             begin = t0[ran].min()
             history.append(n_warps * reads_per_warp * 128 * W / float(t1[ran].max() - begin))
             work = np.diff(ws.astype(np.int64)).astype(np.float64)
-            rate = np.zeros(G)
             finish = np.zeros(G)
             for g in range(G):
                 m = (groups.group_of_sm == g) & ran
                 finish[g] = max(1.0, float(t1[m].max() - begin)) if m.any() else 0.0
-                rate[g] = work[g] / finish[g] if m.any() else 0.0
-            seen = finish[finish > 0]
-            if (seen.max() - seen.min()) / seen.max() <= spread_goal:
+            if finish_spread(finish) <= spread_goal:
                 break
-            rate = np.maximum(rate, rate[rate > 0].min() * 1e-3)
-            weights = np.maximum(1, np.rint(rate / rate.sum() * 1e6)).astype(np.uint32)
+            weights = rebalanced_weights(work, finish)
         win, ws = rr.rr_make_weighted_windows(self.region_bytes, W, weights, n_warps,
                                               max_window_bytes)
         return win, ws, weights, history

@@ -146,3 +146,13 @@ def test_argument_errors():
     with pytest.raises(oracle.OracleError):
         oracle.read_per_sm(1 << 20, 1, 2, 2, 4, seed=1, group_of_sm=np.array([0, 0], np.uint16),
                            windows=np.array([[8000, 1000]], np.uint32))   # window past the region
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+def test_materialised_buffer_read_equals_regenerating_read(W):
+    # 64 MiB really filled and really indexed, against the oracle that regenerates every word
+    n_bytes = (64 << 20) + 256
+    buf = oracle.fill(0, n_bytes // 4)
+    a = oracle.read_logical_materialised(buf, W, 300, 50, seed=11, first_read=3)
+    b = oracle.read_logical(n_bytes, W, 300, 50, seed=11, first_read=3)
+    assert np.array_equal(a, b)
