@@ -96,12 +96,12 @@ int32_t rr_device_info(rr_device_info_t *out /*HOST*/);
  * rr_read_report() decodes.  One scratch buffer must not be shared by calls that overlap.    */
 size_t rr_scratch_bytes(void);
 
-/* ---- A1: fill -----------------------------------------------------------------------------
+/* ---- fill ---------------------------------------------------------------------------------
  * buf[i] = word(i) for i in [0, n_words).  buf: DEVICE, 512-byte aligned, n_words*4 bytes.
  * Asynchronous on `stream`.  n_words = 0 is a no-op.                                          */
 int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
 
-/* ---- A2-A5, A9: random line reads ---------------------------------------------------------
+/* ---- random line reads -------------------------------------------------------------------
  * Paper, Section 2.1 ("every warp reads random coalesced arrays of 32 32-bit words in a memory
  * region of varying size"; 64- and 128-bit words), Section 2.1 second experiment and Section
  * 2.4 (all warps of an SM / of an SM group read inside one chunk).
@@ -217,7 +217,7 @@ int32_t rr_read_block_times(const void *scratch_dev /*DEVICE*/, uint32_t nsm,
 int32_t rr_random_read_static(const rr_read_params_t *params /*HOST*/, void *out_dev /*DEVICE*/,
                               rr_result_t *res /*HOST or NULL*/, void *stream);
 
-/* ---- A6: two-SM contention probe -----------------------------------------------------------
+/* ---- two-SM contention probe ---------------------------------------------------------------
  * Paper, Section 2.2: "if we run our memory access kernel with only two SMs, we expect ... a
  * drop in throughput when those SMs are in the same GPC".  A full grid is launched; blocks exit
  * unless they are the first block on sm_a or sm_b.  Each surviving SM performs total_reads/2
@@ -246,7 +246,7 @@ int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint6
                         float *T_host /*HOST nsm*nsm*/, uint32_t nsm, void *out_dev /*DEVICE*/,
                         void *scratch_dev /*DEVICE*/, double *overlap_min_host, void *stream);
 
-/* ---- A7: contention matrix -> SM groups ----------------------------------------------------
+/* ---- contention matrix -> SM groups --------------------------------------------------------
  * Paper, Section 2.2 and Figure 3 ("rearranging the indices" so groups show as blocks).  Here:
  * symmetrise, quantise against the median, average-linkage agglomeration with exact integer
  * sums, cut at the largest height gap among cuts leaving 2..n/3 clusters, null rule (gap below
@@ -276,7 +276,7 @@ int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratc
 int32_t rr_gpc_map(void *scratch_dev /*DEVICE*/, int32_t *gpc_of_sm_host /*HOST*/,
                    uint32_t *n_gpcs, uint32_t nsm, void *stream);
 
-/* ---- A9 policy: windows per group (host only) ----------------------------------------------
+/* ---- windows per group (host only) -------------------------------------------------------
  * Paper, Section 1.3 ("restricted to a 64GB window (or, say, half the memory for simplicity)")
  * and Section 2.4.  The L lines of the region are cut into K = ceil(L / floor(window_bytes /
  * (128*W))) chunks of floor(L/K) lines, the last running to L.  policy 0: group g takes chunk
@@ -301,7 +301,7 @@ int32_t rr_make_weighted_windows(uint64_t region_bytes, uint32_t words_per_lane,
                                  uint64_t max_window_bytes, rr_window_t *out_host,
                                  uint32_t *warp_start_host);
 
-/* ---- A8: plateau, cliff and reach from a size sweep (host only) ----------------------------
+/* ---- plateau, cliff and reach from a size sweep (host only) --------------------------------
  * Paper, Section 2.1 / Figure 1 ("something dramatic happens when the memory region is larger
  * than about 64GB").  size_bytes strictly increasing.  plateau = lower median of GB/s over
  * 4 GiB <= size <= 32 GiB; a cliff exists iff a larger size has GB/s < 0.8 plateau; reach =

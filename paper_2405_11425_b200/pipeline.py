@@ -105,7 +105,7 @@ class Session:
             raise RuntimeError("allocator returned a buffer that is not 512-byte aligned")
         self.filled = False
 
-    # -- A1 ----------------------------------------------------------------------------------
+    # -- fill --------------------------------------------------------------------------------
     def fill(self) -> float:
         """Fills the whole buffer; returns the write rate in GB/s (CUDA events)."""
         t = self.torch
@@ -117,7 +117,7 @@ class Session:
         self.filled = True
         return self.region_bytes / (e0.elapsed_time(e1) * 1e-3) * 1e-9
 
-    # -- A2-A5, A9 ---------------------------------------------------------------------------
+    # -- reads -------------------------------------------------------------------------------
     def params(self, region_bytes=None, **kw) -> rr.ReadParams:
         kw.setdefault("warps_per_sm", 32)
         kw.setdefault("nsm", self.nsm)
@@ -135,7 +135,7 @@ class Session:
     def checksums(self, n: int) -> np.ndarray:
         return self.out[:n].cpu().numpy().view(np.uint32)
 
-    # -- A8 ----------------------------------------------------------------------------------
+    # -- reach-------------------------------------------------------------------------------
     def size_sweep(self, sizes_bytes, *, seed: int = 7, reads_per_warp: int = 256 * 16, **kw):
         pts = []
         for n in sizes_bytes:
@@ -170,7 +170,7 @@ class Session:
             cliff, plateau, reach = rr.rr_reach([p[0] for p in pts], [p[1] for p in pts])
         return Reach(cliff, plateau, reach, pts)
 
-    # -- A6, A7 ------------------------------------------------------------------------------
+    # -- groups -----------------------------------------------------------------------------
     def discover_groups(self, *, probe_region_bytes=None, total_reads: int = 1 << 18,
                         warps_per_sm: int = 32, seed: int = 5, repeats: int = 3,
                         solo_normalise: bool = True) -> Groups:
@@ -185,7 +185,7 @@ class Session:
         return Groups(g.astype(np.uint16), n_groups, conf, T, overlap, dt,
                       np.bincount(g, minlength=n_groups).tolist())
 
-    # -- A9 ----------------------------------------------------------------------------------
+    # -- windows-------------------------------------------------------------------------------
     def windows(self, groups: Groups, window_bytes: int, W: int = 1, region_bytes=None):
         return rr.rr_make_windows(region_bytes or self.region_bytes, W, window_bytes,
                                   groups.n_groups)

@@ -6,9 +6,9 @@ Experiments (paper section -> BASELINE config):
   size sweep, unrestricted            Section 2.1, Fig. 1            configs[1]
   line widths at 32 GiB               Section 2.1                    configs[2]
   pair probe + clustering             Section 2.2, Fig. 2-3          configs[3]
-  single groups, group pairs          Section 2.3, Fig. 4-5          (next row 1)
+  single groups, group pairs          Section 2.3, Fig. 4-5
   grouped windows over all memory     Section 2.4, Fig. 6            configs[4]
-  sequential reads of the same kernel Section 2.1 ("even better")    (next row 3)
+  sequential reads of the same kernel Section 2.1 ("even better")
 All numbers are event-timed GB/s (10^9 B/s), median of the repetitions; nothing is computed here
 beyond bookkeeping.
 """
@@ -100,7 +100,7 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                     "gpcs_of_group": [sorted(set(gpc[gf.group_of_sm == k].tolist()))
                                       for k in range(gf.n_groups)]}
 
-    # next row 1: every group alone inside the reach, and pairs of groups in distinct windows
+    # Section 2.3: every group alone inside the reach, and pairs of groups in distinct windows
     S = (reach.reach_bytes // 2) if reach.cliff else N // 4
     L_S = S // 128
     singles = []
@@ -254,7 +254,7 @@ def markdown(R: dict) -> str:
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default="gpurun_out/report")
+    ap.add_argument("--out", default="report_out")
     ap.add_argument("--quick", action="store_true")
     a = ap.parse_args(argv)
     R = run(Path(a.out), a.quick)
