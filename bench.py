@@ -7,9 +7,9 @@ Metric (the benchmark spec): random 128-B line read GB/s over the full HBM with every
 to its own window below the measured translation reach, next to the unrestricted rate over the
 same region.  One step = one launch of the persistent read kernel over ~95 % of free HBM:
 148 x 32 logical warps perform 2^8 x 64 random 128-byte line reads each, every warp inside the
-window of the SM group that owns it; windows tile the buffer and both window size and the
-number of warps a group owns follow the group's measured capacity (pooled mode), so that no
-group is the straggler.  The same workload with equal work per SM (the paper's setting) is
+window of the SM that owns it; the windows of one resource group's SMs lie side by side, all
+windows together tile the buffer, and both window size and the number of warps an SM owns follow
+its measured capacity (pooled mode), so that no group is the straggler.  The same workload with equal work per SM (the paper's setting) is
 reported beside it under "calibration".
 
 Before the timed region each rank calibrates its own GPU (the layout differs card to card):
@@ -240,9 +240,12 @@ def run_gpu(args):
     t_bal = time.time()
     n_warps = ses.nsm * WARPS_PER_SM
     max_window = reach.reach_bytes if reach.cliff else 0
+    # one window per SM, side by side inside the SM's resource group (see singleton_groups)
+    owners = ses.singleton_groups(groups)
     bal_windows, warp_start, weights, bal_history = ses.balance(
-        groups, W=1, n_warps=n_warps, reads_per_warp=READS_PER_ITER * ITERS_PER_STEP, seed=SEED,
-        max_window_bytes=max_window, launches_per_round=150, variant=VARIANT_PACKED, unroll=UNROLL)
+        owners, W=1, n_warps=n_warps, reads_per_warp=READS_PER_ITER * ITERS_PER_STEP, seed=SEED,
+        max_window_bytes=max_window, launches_per_round=150, rounds=8, variant=VARIANT_PACKED,
+        unroll=UNROLL)
     t_bal = time.time() - t_bal
     t_cal = time.time() - t_cal
 
@@ -253,7 +256,7 @@ def run_gpu(args):
     def params(step):
         return ses.params(N, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
                           warps_per_sm=WARPS_PER_SM, reads_per_warp=reads, first_read=step * reads,
-                          seed=SEED, group_of_sm=groups.group_of_sm, windows=bal_windows,
+                          seed=SEED, group_of_sm=owners.group_of_sm, windows=bal_windows,
                           warp_start=warp_start, variant=VARIANT_PACKED, unroll=UNROLL)
 
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
@@ -297,7 +300,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
     e2e_seconds = time.perf_counter() - t0
     e2e_bytes, e2e_max = aggregate_throughput(step_bytes * e2e_steps, e2e_seconds)
-    h2d = ses.nsm * 2 + groups.n_groups * 12 + 4 + 128     # tables + scalars in the launch
+    h2d = ses.nsm * 2 + owners.n_groups * 12 + 4 + 128     # tables + scalars in the launch
     d2h = host_out.numel() * 4 + 8208                      # checksums + timing records
 
     # ---- oracle beside it: parity on every warp of a bounded sample, and its timing ---------
@@ -308,7 +311,7 @@ def run_gpu(args):
         oracle.build()
         o_gbps, o_reads, o_dt, o_out = _oracle_sample(N, bal_windows, warp_start, 12.0)
         p = ses.params(N, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps, warps_per_sm=WARPS_PER_SM,
-                       reads_per_warp=o_reads, seed=SEED, group_of_sm=groups.group_of_sm,
+                       reads_per_warp=o_reads, seed=SEED, group_of_sm=owners.group_of_sm,
                        windows=bal_windows, warp_start=warp_start, variant=VARIANT_PACKED,
                        unroll=UNROLL)
         rr.rr_random_read(p, ses.out, ses.scratch)
@@ -334,16 +337,17 @@ def run_gpu(args):
             "ms_per_step": max_seconds / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
             "config": {
-                "workload": "cfg4 grouped full-memory random 128-B line reads: every SM group "
-                            "held to its own window, windows tile the buffer, work and window "
-                            "size in proportion to group capacity, seed 23",
+                "workload": "cfg4 grouped full-memory random 128-B line reads: every SM held to "
+                            "its own window inside its resource group's stretch of the buffer, "
+                            "windows tile the buffer, work and window size in proportion to "
+                            "measured capacity, seed 23",
                 "region_bytes": N, "region_gib": N / GiB, "line_bytes": 128,
                 "logical_warps": n_warps, "warps_per_sm": WARPS_PER_SM,
                 "reads_per_warp_per_step": reads,
                 "kernel": "read_kernel<W=1, U=2, packed>: 8 lanes x 16 B per line, pooled mode",
                 "window_gib_min_max": [float(bal_windows[:, 1].min()) * 128 / GiB,
                                        float(bal_windows[:, 1].max()) * 128 / GiB],
-                "coverage": 1.0, "n_groups": groups.n_groups,
+                "coverage": 1.0, "n_groups": groups.n_groups, "n_windows": owners.n_groups,
                 "l2": "inputs (region) far larger than L2; no flush needed",
                 "parallelism": "replicas" if world > 1 else "single GPU",
             },
@@ -375,8 +379,10 @@ def run_gpu(args):
                           "reach_gib": reach.reach_bytes / GiB,
                           "sweep": [[s / GiB, g] for s, g in reach.sweep]},
                 "balance": {"seconds": t_bal, "gbps_by_round": bal_history,
-                            "weights": weights.tolist(),
-                            "warps_of_group": np.diff(warp_start.astype(np.int64)).tolist()},
+                            "weights_per_sm": weights[owners.group_of_sm].tolist(),
+                            "warps_per_window_min_max": [
+                                int(np.diff(warp_start.astype(np.int64)).min()),
+                                int(np.diff(warp_start.astype(np.int64)).max())]},
                 "equal_work_per_sm": {"window": headline, "window_gib": S / GiB,
                                       "coverage": coverage,
                                       "gbps": window_sweep[headline]["gbps"]},

@@ -274,6 +274,18 @@ class Session:
         rates = sorted(r.gbps for r in res)
         return rates[(len(rates) - 1) // 2], res[-1]
 
+    def singleton_groups(self, groups: Groups) -> Groups:
+        """One "group" per SM, numbered so that the SMs of one resource group are neighbours:
+        their windows then lie side by side inside what would be the resource group's window.
+        A window per SM is still a window per group in the paper's sense (every group's
+        footprint stays below its reach), and it lets each SM's own small translation cache
+        catch a share of the lookups before they reach the group's shared path."""
+        order = np.argsort(groups.group_of_sm, kind="stable")
+        ids = np.empty(self.nsm, dtype=np.uint16)
+        ids[order] = np.arange(self.nsm, dtype=np.uint16)
+        return Groups(ids, self.nsm, groups.confidence, None, groups.overlap_min, 0.0,
+                      [1] * self.nsm)
+
     def naive_control(self, window_bytes: int, seed: int, W: int = 1, region_bytes=None):
         """The paper's per-SM control: every SM on its own picks a pseudo-random chunk."""
         win, cov = rr.rr_make_windows(region_bytes or self.region_bytes, W, window_bytes, self.nsm,

@@ -150,19 +150,35 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                                "windows": rows}
     R["cfg4_grouped"] = cfg4
 
+    # one window per SM, spread over the buffer: how far does an SM's own translation cache reach?
+    MiB = 1 << 20
+    per_sm = []
+    ids = np.arange(ses.nsm, dtype=np.uint16)
+    stride = (N // 128) // ses.nsm
+    for S_sm in (8 * MiB, 32 * MiB, 128 * MiB, 256 * MiB, 512 * MiB, 768 * MiB, 1024 * MiB,
+                 stride * 128):
+        win = np.array([[k * stride, min(S_sm // 128, stride)] for k in range(ses.nsm)], np.uint32)
+        per_sm.append({"window_mib": float(win[0, 1]) * 128 / MiB,
+                       "gbps": _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=ids,
+                                      windows=win)["median"]})
+    R["per_sm_window_sweep"] = per_sm
+
     # work in proportion to group capacity (pooled mode), balanced under sustained load
     balanced = {}
     n_warps = ses.nsm * 32
     max_window = reach.reach_bytes if reach.cliff else 0
-    for W, variant, unroll, name in ((1, rr.RR_VARIANT_PACKED, 2, "128B packed"),
-                                     (1, rr.RR_VARIANT_LDG, 8, "128B 32-lane"),
-                                     (2, rr.RR_VARIANT_LDG, 8, "256B 32-lane")):
-        win, ws, weights, hist = ses.balance(groups, W=W, n_warps=n_warps, reads_per_warp=reads,
+    singles_map = ses.singleton_groups(groups)
+    for W, variant, unroll, owners, name in (
+            (1, rr.RR_VARIANT_PACKED, 2, singles_map, "128B packed, one window per SM"),
+            (1, rr.RR_VARIANT_PACKED, 2, groups, "128B packed, one window per group"),
+            (1, rr.RR_VARIANT_LDG, 8, groups, "128B 32-lane, one window per group"),
+            (2, rr.RR_VARIANT_LDG, 8, groups, "256B 32-lane, one window per group")):
+        win, ws, weights, hist = ses.balance(owners, W=W, n_warps=n_warps, reads_per_warp=reads,
                                              seed=23, max_window_bytes=max_window,
-                                             launches_per_round=20 if quick else 150,
+                                             launches_per_round=20 if quick else 150, rounds=8,
                                              variant=variant, unroll=unroll)
         p = ses.params(N, W=W, mode=rr.RR_MODE_POOLED, n_warps=n_warps, reads_per_warp=reads,
-                       seed=23, group_of_sm=groups.group_of_sm, windows=win, warp_start=ws,
+                       seed=23, group_of_sm=owners.group_of_sm, windows=win, warp_start=ws,
                        variant=variant, unroll=unroll)
         torch.cuda.synchronize()
         time.sleep(1.0)
@@ -242,6 +258,11 @@ def markdown(R: dict) -> str:
             L.append(f"| {name} | {r['window_gib']:.1f} | {r['coverage']:.2f} | {f(r['grouped'])} | "
                      f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} |")
         L.append("")
+    L += ["## One window per SM, windows spread over the buffer (equal work per SM)", "",
+          "| window MiB | GB/s |", "|---|---|"]
+    for r in R.get("per_sm_window_sweep", []):
+        L.append(f"| {r['window_mib']:.0f} | {r['gbps']:.0f} |")
+    L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]
     for name, b in R.get("balanced_pooled", {}).items():

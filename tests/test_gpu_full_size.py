@@ -189,3 +189,24 @@ def test_pooled_bench_launch_configuration_sampled(ses):
                                                      n), v
     t0, t1 = rr.rr_read_block_times(ses.scratch, ses.nsm)
     assert (t1 > t0).all() and t0.min() > 0
+
+
+def test_pooled_one_window_per_sm_sampled(ses):
+    # bench.py's owner map: one window per SM (148 "groups"), weights differing per SM
+    region = ses.region_bytes
+    rng = np.random.default_rng(3)
+    owners = rng.permutation(ses.nsm).astype(np.uint16)
+    weights = rng.integers(5000, 8000, ses.nsm)
+    n_warps = ses.nsm * WPS
+    win, ws = rr.rr_make_weighted_windows(region, 1, weights, n_warps, max_window_bytes=64 * GiB)
+    reads = 256 * 64
+    p = ses.params(region, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps, warps_per_sm=WPS,
+                   reads_per_warp=reads, seed=rr_inputs.CFG4_SEED, group_of_sm=owners, windows=win,
+                   warp_start=ws, variant=rr.RR_VARIANT_PACKED, unroll=2)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == ses.nsm
+    got = ses.checksums(n_warps)
+    for v in _sample(n_warps):
+        g = int(np.searchsorted(ws, v, side="right") - 1)
+        base, n = map(int, win[g])
+        assert tuple(got[v]) == oracle.warp_checksum(rr_inputs.CFG4_SEED, v, 0, reads, 1, base, n), v
