@@ -210,3 +210,30 @@ def test_pooled_one_window_per_sm_sampled(ses):
         g = int(np.searchsorted(ws, v, side="right") - 1)
         base, n = map(int, win[g])
         assert tuple(got[v]) == oracle.warp_checksum(rr_inputs.CFG4_SEED, v, 0, reads, 1, base, n), v
+
+
+def test_balancing_loop_yields_a_valid_plan_and_exact_checksums(ses):
+    # Session.balance on the card's real groups: whatever weights the timers lead to, the plan
+    # must tile the buffer, hand out every logical warp once, and the read must stay bit exact
+    groups = ses.discover_groups(total_reads=1 << 16, repeats=3)
+    owners = ses.singleton_groups(groups)
+    assert sorted(owners.group_of_sm.tolist()) == list(range(ses.nsm))
+    order = np.argsort(owners.group_of_sm)          # SMs in window order: resource groups contiguous
+    assert (np.diff(groups.group_of_sm[order].astype(np.int64)) >= 0).all()
+    n_warps = ses.nsm * WPS
+    win, ws, weights, history = ses.balance(owners, n_warps=n_warps, reads_per_warp=4096,
+                                            rounds=3, launches_per_round=3,
+                                            variant=rr.RR_VARIANT_PACKED, unroll=2)
+    L = ses.region_bytes // 128
+    assert win[0, 0] == 0 and int(win[-1, 0]) + int(win[-1, 1]) == L
+    assert np.array_equal(win[1:, 0], win[:-1, 0] + win[:-1, 1])
+    assert ws[0] == 0 and ws[-1] == n_warps and (np.diff(ws.astype(np.int64)) > 0).all()
+    assert len(history) >= 1 and all(h > 100 for h in history) and weights.min() >= 1
+    rate, res = ses.read_pooled(owners, win, ws, reads_per_warp=4096, seed=23,
+                                variant=rr.RR_VARIANT_PACKED, unroll=2)
+    assert res.sms_covered == ses.nsm and rate > 100
+    got = ses.checksums(n_warps)
+    for v in _sample(n_warps):
+        g = int(np.searchsorted(ws, v, side="right") - 1)
+        base, n = map(int, win[g])
+        assert tuple(got[v]) == oracle.warp_checksum(23, v, 0, 4096, 1, base, n), v
