@@ -61,6 +61,13 @@ def _load():
         lib.orc_line.argtypes = [u32, u64, u64, u64, u64, u64, u64]
         lib.orc_warp_checksum.restype = None
         lib.orc_warp_checksum.argtypes = [u32, u64, u64, u64, u64, u64, u32, u64, u64, p, p]
+        lib.orc_line_phased.restype = u64
+        lib.orc_line_phased.argtypes = [u64, u64, u64, u64, u64, u64, u64]
+        lib.orc_warp_checksum_phased.restype = None
+        lib.orc_warp_checksum_phased.argtypes = [u64, u64, u64, u64, u32, u64, u64, u64, u64, p, p]
+        lib.orc_read_per_sm_phased.restype = i32
+        lib.orc_read_per_sm_phased.argtypes = [u64, u32, u32, u32, u64, u64, u64, p, p, p, u32, u64,
+                                               u64, p]
         lib.orc_read_logical.restype = i32
         lib.orc_read_logical.argtypes = [u64, u32, u32, u64, u64, u64, u64, p]
         lib.orc_read_logical_materialised.restype = i32
@@ -169,6 +176,42 @@ def read_per_sm(region_bytes: int, W: int, nsm: int, wps: int, reads: int, seed:
         ng = w.shape[0]
     rc = _load().orc_read_per_sm(region_bytes, W, index_mode, nsm, wps, first_read, reads, seed,
                                  _ptr(g), _ptr(wb), _ptr(wn), ng, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def line_phased(seed: int, v: int, i: int, base: int, n: int, phase_reads: int,
+                sub_lines: int) -> int:
+    return int(_load().orc_line_phased(seed, v, i, base, n, phase_reads, sub_lines))
+
+
+def warp_checksum_phased(seed: int, v: int, first_read: int, reads: int, W: int, base: int, n: int,
+                         phase_reads: int, sub_lines: int):
+    x = ctypes.c_uint32()
+    s = ctypes.c_uint32()
+    _load().orc_warp_checksum_phased(seed, v, first_read, reads, W, base, n, phase_reads, sub_lines,
+                                     ctypes.byref(x), ctypes.byref(s))
+    return int(x.value), int(s.value)
+
+
+def read_per_sm_phased(region_bytes: int, W: int, nsm: int, wps: int, reads: int, seed: int,
+                       phase_reads: int, phase_window_bytes: int, group_of_sm=None, windows=None,
+                       first_read: int = 0) -> np.ndarray:
+    """Per-SM mode with windows that move: phase p of a warp's stream reads inside sub-window
+    p mod Q of the warp's window."""
+    out = np.zeros((nsm * wps, 2), dtype=np.uint32)
+    g = wb = wn = None
+    ng = 0
+    if group_of_sm is not None:
+        g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+        w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+        wb = np.ascontiguousarray(w[:, 0])
+        wn = np.ascontiguousarray(w[:, 1])
+        ng = w.shape[0]
+    rc = _load().orc_read_per_sm_phased(region_bytes, W, nsm, wps, first_read, reads, seed, _ptr(g),
+                                        _ptr(wb), _ptr(wn), ng, phase_reads, phase_window_bytes,
+                                        _ptr(out))
     if rc != 0:
         raise OracleError(rc)
     return out

@@ -123,7 +123,83 @@ void orc_warp_checksum(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t 
     *S = s;
 }
 
+/* ---- O3b: windows that move with time ------------------------------------------
+ * Section 1.3 asks that "any particular warp only accesses a smaller region"; the
+ * paper fixes that region for good.  Reading for hardware whose per-SM translation
+ * cache is smaller than its share of memory: the warp's window of n lines is cut into
+ * Q = ceil(n / sub_lines) sub-windows [floor(n q / Q), floor(n (q+1) / Q)); reads come
+ * in phases of phase_reads reads, phase p = floor(i / phase_reads) of a warp's stream
+ * (i = absolute read counter) draws uniformly inside sub-window p mod Q.  Over Q
+ * phases every line of the window is equally likely; at any moment a warp is held to
+ * n/Q lines.  With sub_lines >= n this is the plain random mode.                    */
+uint64_t orc_line_phased(uint64_t seed, uint64_t v, uint64_t i, uint64_t base, uint64_t n,
+                         uint64_t phase_reads, uint64_t sub_lines)
+{
+    uint64_t Q = (n + sub_lines - 1) / sub_lines;
+    uint64_t q = (i / phase_reads) % Q;
+    uint64_t lo = n * q / Q, hi = n * (q + 1) / Q; /* n < 2^32, Q <= n: fits 64 bits */
+    return base + lo + orc_draw(seed, v, i) % (hi - lo);
+}
+
+void orc_warp_checksum_phased(uint64_t seed, uint64_t v, uint64_t first_read, uint64_t reads,
+                              uint32_t W, uint64_t base, uint64_t n, uint64_t phase_reads,
+                              uint64_t sub_lines, uint32_t *X, uint32_t *S)
+{
+    uint32_t x = 0, s = 0;
+    for (uint64_t t = 0; t < reads; ++t) {
+        uint64_t line = orc_line_phased(seed, v, first_read + t, base, n, phase_reads, sub_lines);
+        for (uint32_t lane = 0; lane < 32; ++lane)
+            for (uint32_t w = 0; w < W; ++w) {
+                uint32_t word = orc_word(line * 32u * W + (uint64_t)lane * W + w);
+                x ^= word;
+                s += word;
+            }
+    }
+    *X = x;
+    *S = s;
+}
+
 static int orc_width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
+
+/* Per-SM mode with moving windows (see orc_line_phased); arguments as orc_read_per_sm.
+ * nsm = 0 with group_of_sm = NULL is not accepted; for logical warps over the whole
+ * region pass one group covering everything.                                        */
+int32_t orc_read_per_sm_phased(uint64_t region_bytes, uint32_t W, uint32_t nsm, uint32_t wps,
+                               uint64_t first_read, uint64_t reads, uint64_t seed,
+                               const uint16_t *group_of_sm, const uint32_t *win_base,
+                               const uint32_t *win_n, uint32_t n_groups, uint64_t phase_reads,
+                               uint64_t phase_window_bytes, uint32_t *out)
+{
+    if (!orc_width_ok(W) || !out || nsm == 0 || wps == 0 || phase_reads == 0) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    uint64_t sub = phase_window_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull || sub == 0) return ORC_ERR_RANGE;
+    if (group_of_sm) {
+        if (!win_base || !win_n || n_groups == 0) return ORC_ERR_ARG;
+        for (uint32_t g = 0; g < n_groups; ++g)
+            if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
+        for (uint32_t s = 0; s < nsm; ++s)
+            if (group_of_sm[s] != ORC_SM_INACTIVE && group_of_sm[s] >= n_groups) return ORC_ERR_MAP;
+    }
+    int64_t nw = (int64_t)nsm * wps;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t sm = (uint32_t)(v / wps);
+        uint64_t base = 0, n = L;
+        if (group_of_sm) {
+            if (group_of_sm[sm] == ORC_SM_INACTIVE) {
+                out[2 * v] = 0;
+                out[2 * v + 1] = 0;
+                continue;
+            }
+            base = win_base[group_of_sm[sm]];
+            n = win_n[group_of_sm[sm]];
+        }
+        orc_warp_checksum_phased(seed, (uint64_t)v, first_read, reads, W, base, n, phase_reads, sub,
+                                 &out[2 * v], &out[2 * v + 1]);
+    }
+    return ORC_OK;
+}
 
 /* The same logical-mode read performed on a real buffer in host memory (filled with
  * orc_fill): the line is indexed literally instead of regenerated.  This is the CPU
