@@ -247,6 +247,24 @@ def run_gpu(args):
         max_window_bytes=max_window, launches_per_round=150, rounds=8, variant=VARIANT_PACKED,
         unroll=UNROLL)
     t_bal = time.time() - t_bal
+
+    # the same slices with windows that move (phased index): every SM works through its slice in
+    # eight sub-windows, one per 1024 reads, so that its own translation cache holds the live part
+    mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
+    mv_sub = (int(mv_windows[:, 1].max()) * 128 + 7) // 8
+    mv = ses.params(N, W=1, warps_per_sm=WARPS_PER_SM, reads_per_warp=READS_PER_ITER * ITERS_PER_STEP,
+                    seed=SEED, group_of_sm=owners.group_of_sm, windows=mv_windows,
+                    variant=VARIANT_PACKED, unroll=UNROLL, index_mode=rr.RR_INDEX_PHASED,
+                    phase_reads=1024, phase_window_bytes=mv_sub)
+    for _ in range(SETTLE_LAUNCHES):
+        rr.rr_random_read(mv, ses.out, ses.scratch, timed=False)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(100):
+        rr.rr_random_read(mv, ses.out, ses.scratch, timed=False)
+    ev1.record()
+    torch.cuda.synchronize()
+    moving_gbps = rr.rr_read_report(mv, ses.scratch).bytes * 100 / ev0.elapsed_time(ev1) * 1e-6
     t_cal = time.time() - t_cal
 
     # ---- timed region: device-resident, asynchronous launches -------------------------------
@@ -383,6 +401,10 @@ def run_gpu(args):
                             "warps_per_window_min_max": [
                                 int(np.diff(warp_start.astype(np.int64)).min()),
                                 int(np.diff(warp_start.astype(np.int64)).max())]},
+                "moving_windows": {"gbps_sustained": moving_gbps, "phase_reads": 1024,
+                                   "sub_window_mib": mv_sub / (1 << 20), "sub_windows": 8,
+                                   "note": "same per-SM slices, equal work per SM, each SM held "
+                                           "to one eighth of its slice at a time"},
                 "equal_work_per_sm": {"window": headline, "window_gib": S / GiB,
                                       "coverage": coverage,
                                       "gbps": window_sweep[headline]["gbps"]},

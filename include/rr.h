@@ -25,6 +25,10 @@
  *   r(seed,v,i)  = sm64(k_v + i * 0x9E3779B97F4A7C15)      -- i-th draw of warp v
  *   line(v,i)    = base + (r mod n)   for a window of n lines starting at line `base`
  *                  (RR_INDEX_STRIDE: base + ((i * V + v) mod n), V = warps in the call)
+ *                  (RR_INDEX_PHASED: the window is cut into Q = ceil(n / sub) sub-windows
+ *                  [floor(n q / Q), floor(n (q+1) / Q)), sub = phase_window_bytes / (128 W);
+ *                  read i belongs to phase p = floor(i / phase_reads) and draws
+ *                  base + lo_q + (r mod (hi_q - lo_q)) with q = p mod Q)
  *   checksum     = {X, S}: X = xor, S = sum mod 2^32 of every 32-bit word the warp read
  */
 #ifndef RR_H_
@@ -63,6 +67,7 @@ extern "C" {
 #define RR_MODE_POOLED 2u  /* logical warps owned by SM groups; the group's SMs share the work  */
 #define RR_INDEX_RANDOM 0u
 #define RR_INDEX_STRIDE 1u
+#define RR_INDEX_PHASED 2u /* random inside a sub-window that moves with the read counter         */
 #define RR_VARIANT_LDG 0u         /* ld.global.nc.L1::no_allocate vector loads                  */
 #define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
 #define RR_VARIANT_PACKED 2u      /* every lane loads 16 bytes: one warp load covers 4/W lines  */
@@ -126,6 +131,10 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   groups' capacities (rr_make_weighted_windows).  out has n_warps entries, accumulated with
  *   atomics (the call clears it first); the checksums do not depend on which SM did what.
  *   Every group that owns warps needs at least one active SM, else RR_ERR_MAP.
+ * RR_INDEX_PHASED (LOGICAL and PER_SM modes; first_read must be a multiple of 32): Section 1.3
+ *   wants each warp held to a smaller region; here that region also moves, so that an SM whose
+ *   own translation cache is smaller than its share of memory works through its window one
+ *   sub-window at a time while a whole cycle of phases still covers the window uniformly.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
@@ -159,6 +168,9 @@ typedef struct {
     uint32_t unroll;
     uint32_t pool_block_reads;  /* POOLED: smallest grab in reads, 0 = 64; else must be 0      */
     const uint32_t *warp_start; /* POOLED: HOST [n_groups+1]; else NULL                        */
+    uint32_t phase_reads;       /* RR_INDEX_PHASED: reads per phase, a power of two >= 32      */
+    uint32_t reserved;          /* must be 0                                                   */
+    uint64_t phase_window_bytes; /* RR_INDEX_PHASED: largest sub-window                        */
 } rr_read_params_t;
 
 typedef struct {

@@ -22,7 +22,7 @@ RR_ERR_STATIC_LIMIT = -10
 RR_STATIC_MAX_SM, RR_STATIC_SCRATCH_BYTES = 192, 5888
 RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0xFFFF
 RR_MODE_LOGICAL, RR_MODE_PER_SM, RR_MODE_POOLED = 0, 1, 2
-RR_INDEX_RANDOM, RR_INDEX_STRIDE = 0, 1
+RR_INDEX_RANDOM, RR_INDEX_STRIDE, RR_INDEX_PHASED = 0, 1, 2
 RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED, RR_VARIANT_PACKED = 0, 1, 2
 
 EXPORTS = (
@@ -59,6 +59,8 @@ class _ReadParams(ctypes.Structure):
         ("windows", ctypes.c_void_p), ("n_groups", ctypes.c_uint32),
         ("variant", ctypes.c_uint32), ("unroll", ctypes.c_uint32),
         ("pool_block_reads", ctypes.c_uint32), ("warp_start", ctypes.c_void_p),
+        ("phase_reads", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("phase_window_bytes", ctypes.c_uint64),
     ]
 
 
@@ -205,7 +207,8 @@ class ReadParams:
                  index_mode: int = RR_INDEX_RANDOM, n_warps: int = 0, warps_per_sm: int = 32,
                  nsm: int = 0, reads_per_warp: int = 0, first_read: int = 0, seed: int = 0,
                  group_of_sm=None, windows=None, variant: int = RR_VARIANT_LDG, unroll: int = 0,
-                 warp_start=None, pool_block_reads: int = 0):
+                 warp_start=None, pool_block_reads: int = 0, phase_reads: int = 0,
+                 phase_window_bytes: int = 0):
         self._groups = None
         self._windows = None
         self._warp_start = None
@@ -224,7 +227,8 @@ class ReadParams:
             self._groups.ctypes.data if self._groups is not None else None,
             self._windows.ctypes.data if self._windows is not None else None,
             n_groups, variant, unroll, pool_block_reads,
-            self._warp_start.ctypes.data if self._warp_start is not None else None)
+            self._warp_start.ctypes.data if self._warp_start is not None else None,
+            phase_reads, 0, phase_window_bytes)
 
 
 def _result(r: _Result) -> ReadResult:

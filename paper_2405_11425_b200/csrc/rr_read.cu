@@ -23,13 +23,51 @@ struct Tables {
     uint32_t warp_start[RR_MAX_GROUPS + 1];  // POOLED
 };
 
+// How read i of a warp's stream picks its line inside the warp's window.
+struct IndexSpec {
+    uint32_t mode;         // RR_INDEX_*
+    uint32_t phase_shift;  // PHASED: log2(reads per phase)
+    uint32_t sub_lines;    // PHASED: largest sub-window, in lines
+};
+
+// The window a batch of 32 reads draws from: the warp's whole window, or (PHASED) the
+// sub-window of the batch's phase.  Recomputed only when the phase changes.
+struct LineSource {
+    uint32_t base;
+    Divisor div;
+    uint32_t win_base, win_n;
+    uint64_t n_sub, phase;
+    __device__ __forceinline__ void init(uint32_t b, uint32_t n, const IndexSpec &ix)
+    {
+        win_base = base = b;
+        win_n = n;
+        div = make_divisor(n);
+        phase = ~0ull;
+        n_sub = ix.mode == RR_INDEX_PHASED ? ((uint64_t)n + ix.sub_lines - 1) / ix.sub_lines : 1;
+    }
+    // i0 = absolute index of the first read of a batch; all 32 reads of a batch share a phase
+    // because phases are multiples of 32 reads and streams start at multiples of 32
+    __device__ __forceinline__ void enter(uint64_t i0, const IndexSpec &ix)
+    {
+        if (ix.mode != RR_INDEX_PHASED) return;
+        const uint64_t p = i0 >> ix.phase_shift;
+        if (p == phase) return;
+        phase = p;
+        const uint64_t q = p % n_sub;
+        const uint64_t lo = (uint64_t)win_n * q / n_sub, hi = (uint64_t)win_n * (q + 1) / n_sub;
+        base = win_base + (uint32_t)lo;
+        div = make_divisor((uint32_t)(hi - lo));
+    }
+};
+
 struct ReadArgs {
     const char *buf;
     uint64_t region_bytes;
     uint64_t reads, first_read;
     uint64_t key_seed;  // sm64(seed)
     uint32_t n_lines;   // L of the whole region
-    uint32_t mode, index_mode;
+    uint32_t mode;
+    IndexSpec ix;
     uint32_t n_warps;        // LOGICAL
     uint32_t wps, wpc, cps;  // warps per SM, per block; blocks per SM
     uint32_t nsm;
@@ -43,20 +81,21 @@ constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2;
 
 template <int W, int U, bool CHECKED>
 __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, uint64_t region_bytes,
-                                           uint64_t key, uint32_t index_mode, uint64_t v,
+                                           uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
                                            uint32_t &S, uint32_t *violations)
 {
     static_assert(U >= 1 && U <= 16 && (32 % U) == 0, "ring depth must divide a batch");
-    const Divisor div = make_divisor(n);
+    LineSource src;
+    src.init(base, n, ix);
     const char *lane_ptr = buf + lane * (4u * W);
     uint32_t d[U][W];
     uint32_t x = 0, s = 0;
 
     auto gen = [&](uint64_t i) -> uint32_t {
-        uint64_t r = (index_mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
-        return base + mod_exact(r, div);
+        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[W]) {
         if (CHECKED) {
@@ -80,6 +119,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
     };
 
     const uint64_t n_batches = (reads + 31) >> 5;
+    src.enter(first, ix);
     uint32_t cur = gen(first + lane);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -93,6 +133,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
     }
     for (uint64_t b = 0; b < n_batches; ++b) {
         const uint64_t t0 = b << 5;
+        src.enter(first + t0 + 32, ix);
         const uint32_t nxt = gen(first + t0 + 32 + lane);
         if (t0 + 32 + U <= reads) {  // every read of this batch and its refills exist
 #pragma unroll
@@ -129,7 +170,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
 // workload runs into the board's power limit and every instruction not issued buys clock.
 template <int W, int U>
 __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, uint64_t key,
-                                                  uint32_t index_mode, uint64_t v, uint64_t V,
+                                                  IndexSpec ix, uint64_t v, uint64_t V,
                                                   uint64_t first, uint64_t reads, uint32_t base,
                                                   uint32_t n, uint32_t lane, uint32_t &X,
                                                   uint32_t &S)
@@ -138,15 +179,16 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     constexpr int NL = 32 / P;   // warp loads per batch of 32 reads = lanes per line
     static_assert(W == 1 || W == 2, "16-byte lanes already cover a 512-byte line");
     static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a batch");
-    const Divisor div = make_divisor(n);
+    LineSource src;
+    src.init(base, n, ix);
     const uint32_t sub = lane / NL;  // which of the P lines of a load this lane serves
     const char *lane_ptr = buf + (lane % NL) * 16u;
     uint32_t d[U][4];
     uint32_t x = 0, s = 0;
 
     auto gen = [&](uint64_t i) -> uint32_t {
-        uint64_t r = (index_mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
-        return base + mod_exact(r, div);
+        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[4]) {
         load_lane<4>(lane_ptr + (uint64_t)line * (128u * W), dst);
@@ -160,6 +202,7 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     };
 
     const uint64_t n_batches = (reads + 31) >> 5;
+    src.enter(first, ix);
     uint32_t cur = gen(first + lane);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -168,6 +211,7 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     }
     for (uint64_t b = 0; b < n_batches; ++b) {
         const uint64_t t0 = b << 5;
+        src.enter(first + t0 + 32, ix);
         const uint32_t nxt = gen(first + t0 + 32 + lane);
         if (t0 + 32 + U * P <= reads) {  // every read of this batch and its refills exist
 #pragma unroll
@@ -202,15 +246,15 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
 
 template <int W, int U, int VAR>
 __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
-                                           uint64_t key, uint32_t index_mode, uint64_t v,
+                                           uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
                                            uint32_t &S, uint32_t *violations)
 {
     if constexpr (VAR == kVarPacked && W < 4)
-        warp_reads_packed<W, U>(buf, key, index_mode, v, V, first, reads, base, n, lane, X, S);
+        warp_reads_packed<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S);
     else
-        warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, index_mode, v, V, first,
+        warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, ix, v, V, first,
                                                    reads, base, n, lane, X, S, violations);
 }
 
@@ -279,7 +323,7 @@ __global__ void __launch_bounds__(1024, 1)
                 const uint64_t n_seg = (end - x < a.reads - i0) ? end - x : a.reads - i0;
                 const uint64_t v = v0 + w;
                 uint32_t X, S;
-                warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode,
+                warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix,
                                           v, a.n_warps, a.first_read + i0, n_seg, base, n, lane, X,
                                           S, &sc->violations);
                 if (lane == 0) {
@@ -323,7 +367,7 @@ __global__ void __launch_bounds__(1024, 1)
         const uint64_t v = (uint64_t)sm * a.wps + slot * a.wpc + warp;
         const uint64_t V = (uint64_t)a.nsm * a.wps;
         uint32_t X, S;
-        warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v, V,
+        warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v, V,
                                   a.first_read, a.reads, base, n, lane, X, S, &sc->violations);
         if (lane == 0) a.out[v] = make_uint2(X, S);
         __syncthreads();
@@ -342,7 +386,7 @@ __global__ void __launch_bounds__(1024, 1)
         const uint64_t stride = (uint64_t)gridDim.x * a.wpc;
         for (uint64_t v = (uint64_t)blockIdx.x * a.wpc + warp; v < a.n_warps; v += stride) {
             uint32_t X, S;
-            warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.index_mode, v,
+            warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
                                       a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
                                       &sc->violations);
             if (lane == 0) a.out[v] = make_uint2(X, S);
@@ -394,7 +438,8 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     const uint64_t v = (uint64_t)sm * a.wps + warp;
     uint32_t X, S;
     warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
-                                       RR_INDEX_RANDOM, v, (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
+                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u}, v,
+                                       (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
                                        a.n_lines, lane, X, S, nullptr);
     if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
     __syncthreads();
@@ -453,8 +498,16 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
 {
     if (!p || !out || !scratch || !p->buf) return RR_ERR_ARG;
     if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_POOLED ||
-        p->index_mode > RR_INDEX_STRIDE || p->variant > RR_VARIANT_PACKED)
+        p->index_mode > RR_INDEX_PHASED || p->variant > RR_VARIANT_PACKED)
         return RR_ERR_ARG;
+    if (p->reserved) return RR_ERR_ARG;
+    if (p->index_mode == RR_INDEX_PHASED) {
+        const uint32_t b = p->phase_reads;
+        if (b < 32 || (b & (b - 1)) || p->first_read % 32u) return RR_ERR_ARG;
+        if (p->phase_window_bytes < 128ull * p->words_per_lane) return RR_ERR_RANGE;
+    } else if (p->phase_reads || p->phase_window_bytes) {
+        return RR_ERR_ARG;
+    }
     if (p->mode != RR_MODE_POOLED && (p->pool_block_reads || p->warp_start)) return RR_ERR_ARG;
     uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_PACKED ? 4u : 8u);
     if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && p->variant == RR_VARIANT_PACKED))
@@ -643,7 +696,14 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     a.key_seed = sm64(p->seed);
     a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
     a.mode = p->mode;
-    a.index_mode = p->index_mode;
+    a.ix.mode = p->index_mode;
+    a.ix.phase_shift = 0;
+    a.ix.sub_lines = 0;
+    if (p->index_mode == RR_INDEX_PHASED) {
+        while ((1u << a.ix.phase_shift) < p->phase_reads) ++a.ix.phase_shift;
+        const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
+        a.ix.sub_lines = sub > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sub;
+    }
     a.n_warps = p->n_warps;
     a.wps = g.wps;
     a.wpc = g.wpc;
@@ -1016,7 +1076,14 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     a.key_seed = sm64(p->seed);
     a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
     a.mode = p->mode;
-    a.index_mode = p->index_mode;
+    a.ix.mode = p->index_mode;
+    a.ix.phase_shift = 0;
+    a.ix.sub_lines = 0;
+    if (p->index_mode == RR_INDEX_PHASED) {
+        while ((1u << a.ix.phase_shift) < p->phase_reads) ++a.ix.phase_shift;
+        const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
+        a.ix.sub_lines = sub > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sub;
+    }
     a.n_warps = p->n_warps;
     a.wps = g.wps;
     a.wpc = g.wpc;

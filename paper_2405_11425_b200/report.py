@@ -163,6 +163,32 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                                       windows=win)["median"]})
     R["per_sm_window_sweep"] = per_sm
 
+    # moving windows: every SM owns 1/148 of the buffer and works through it in sub-windows
+    owners_eq = ses.singleton_groups(groups)
+    eq_win, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, ses.nsm * 32)
+    slice_bytes = int(eq_win[:, 1].max()) * 128
+    moving = []
+    for parts in (2, 4, 8, 16):
+        for B in (256, 1024, 4096):
+            p = ses.params(N, seed=23, reads_per_warp=reads, group_of_sm=owners_eq.group_of_sm,
+                           windows=eq_win, variant=rr.RR_VARIANT_PACKED, unroll=2,
+                           index_mode=rr.RR_INDEX_PHASED, phase_reads=B,
+                           phase_window_bytes=(slice_bytes + parts - 1) // parts)
+            n = 30 if quick else 200
+            for _ in range(10 if quick else 100):
+                rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+            e1.record()
+            torch.cuda.synchronize()
+            rep = rr.rr_read_report(p, ses.scratch)
+            moving.append({"sub_windows": parts, "sub_window_mib": slice_bytes / parts / MiB,
+                           "phase_reads": B,
+                           "sustained_gbps": rep.bytes * n / e0.elapsed_time(e1) * 1e-6})
+    R["moving_windows"] = moving
+
     # work in proportion to group capacity (pooled mode), balanced under sustained load
     balanced = {}
     n_warps = ses.nsm * 32
@@ -262,6 +288,12 @@ def markdown(R: dict) -> str:
           "| window MiB | GB/s |", "|---|---|"]
     for r in R.get("per_sm_window_sweep", []):
         L.append(f"| {r['window_mib']:.0f} | {r['gbps']:.0f} |")
+    L.append("")
+    L += ["## Moving windows: one slice per SM, read one sub-window at a time (sustained GB/s)", "",
+          "| sub-windows per slice | sub-window MiB | reads per phase | GB/s |", "|---|---|---|---|"]
+    for r in R.get("moving_windows", []):
+        L.append(f"| {r['sub_windows']} | {r['sub_window_mib']:.0f} | {r['phase_reads']} | "
+                 f"{r['sustained_gbps']:.0f} |")
     L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]

@@ -175,6 +175,20 @@ def test_pooled_mode_argument_errors():
     assert _call(warp_start=[0, 4]) == rr.RR_ERR_ARG
 
 
+def test_phased_index_argument_errors():
+    ok = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=256, phase_window_bytes=1 << 16)
+    assert _call(**{**ok, "phase_reads": 0}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "phase_reads": 16}) == rr.RR_ERR_ARG
+    assert _call(**{**ok, "phase_reads": 96}) == rr.RR_ERR_ARG            # not a power of two
+    assert _call(**{**ok, "first_read": 5}) == rr.RR_ERR_ARG              # streams start at x32
+    assert _call(**{**ok, "phase_window_bytes": 64}) == rr.RR_ERR_RANGE
+    assert _call(phase_reads=256) == rr.RR_ERR_ARG                        # only with PHASED
+    assert _call(phase_window_bytes=1 << 20) == rr.RR_ERR_ARG
+    g = np.array([0, 1, 0, 1], np.uint16)
+    assert _call(mode=rr.RR_MODE_POOLED, n_warps=10, nsm=4, warps_per_sm=8, group_of_sm=g,
+                 windows=[[0, 100], [100, 100]], warp_start=[0, 4, 10], **ok) == rr.RR_ERR_ARG
+
+
 def test_reach_matches_oracle():
     rng = np.random.default_rng(3)
     sizes = [s << 30 for s in (1, 4, 16, 32, 48, 64, 96, 128, 160, 169)]

@@ -237,3 +237,24 @@ def test_balancing_loop_yields_a_valid_plan_and_exact_checksums(ses):
         g = int(np.searchsorted(ws, v, side="right") - 1)
         base, n = map(int, win[g])
         assert tuple(got[v]) == oracle.warp_checksum(23, v, 0, 4096, 1, base, n), v
+
+
+def test_moving_windows_over_the_whole_buffer_sampled(ses):
+    # one slice of the buffer per SM, eight sub-windows per slice, 1024 reads per phase
+    region = ses.region_bytes
+    rng = np.random.default_rng(5)
+    owners = rng.permutation(ses.nsm).astype(np.uint16)
+    win, _ = rr.rr_make_weighted_windows(region, 1, [1] * ses.nsm, ses.nsm * WPS)
+    sub_bytes = (int(win[:, 1].max()) * 128 + 7) // 8
+    reads, first = 256 * 64, 256 * 64 * 2
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=reads, first_read=first,
+                   seed=rr_inputs.CFG4_SEED, group_of_sm=owners, windows=win,
+                   variant=rr.RR_VARIANT_PACKED, unroll=2, index_mode=rr.RR_INDEX_PHASED,
+                   phase_reads=1024, phase_window_bytes=sub_bytes)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == ses.nsm and res.bytes == ses.nsm * WPS * reads * 128
+    got = ses.checksums(ses.nsm * WPS)
+    for v in _sample(ses.nsm * WPS):
+        base, n = map(int, win[owners[v // WPS]])
+        assert tuple(got[v]) == oracle.warp_checksum_phased(rr_inputs.CFG4_SEED, v, first, reads, 1,
+                                                            base, n, 1024, sub_bytes // 128), v

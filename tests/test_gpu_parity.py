@@ -348,3 +348,36 @@ def test_packed_variant_grouped_pooled_and_stride(dev, W):
     rr.rr_random_read(p, out, dev.scratch)
     assert np.array_equal(_np(out), oracle.read_logical(small, W, V, R, 0,
                                                         index_mode=oracle.INDEX_STRIDE))
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+@pytest.mark.parametrize("variant", [rr.RR_VARIANT_LDG, rr.RR_VARIANT_PACKED,
+                                     rr.RR_VARIANT_LDG_CHECKED])
+def test_phased_index_mode_matches_oracle(dev, W, variant):
+    region = dev.buf_bytes
+    G = 5
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=6, inactive_frac=0.05)
+    windows, _ = rr.rr_make_windows(region, W, region // 5, G)
+    windows[1] = (777, 10007)                       # sub-windows of unequal size
+    for B, sub_bytes, reads, first in [(32, 1000 * 128 * W, 300, 0), (64, 3000 * 128 * W, 129, 64),
+                                       (256, 8 << 20, 1000, 32 * 9), (1024, 1 << 40, 100, 0)]:
+        out = _out(dev, dev.nsm * 8)
+        p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=8, reads_per_warp=reads,
+                          first_read=first, seed=23, group_of_sm=groups, windows=windows,
+                          variant=variant, index_mode=rr.RR_INDEX_PHASED, phase_reads=B,
+                          phase_window_bytes=sub_bytes)
+        res = rr.rr_random_read(p, out, dev.scratch)
+        assert res.violations == 0
+        expect = oracle.read_per_sm_phased(region, W, dev.nsm, 8, reads, 23, B, sub_bytes,
+                                           group_of_sm=groups, windows=windows, first_read=first)
+        assert np.array_equal(_np(out), expect), (W, variant, B, sub_bytes, reads, first)
+    # logical mode: one window = the region (compare through a one-group per-SM oracle call)
+    L = region // (128 * W)
+    out = _out(dev, 64)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=64, reads_per_warp=200,
+                      seed=3, variant=variant, index_mode=rr.RR_INDEX_PHASED, phase_reads=32,
+                      phase_window_bytes=64 << 20)
+    rr.rr_random_read(p, out, dev.scratch)
+    expect = oracle.read_per_sm_phased(region, W, 2, 32, 200, 3, 32, 64 << 20,
+                                       group_of_sm=np.zeros(2, np.uint16), windows=[[0, L]])
+    assert np.array_equal(_np(out), expect)
