@@ -624,6 +624,43 @@ static int32_t ballast_for_occupancy(K kernel, int block, int want, const Device
     return RR_ERR_CUDA;
 }
 
+// Kernel arguments of one read launch from the caller's parameters and the launch geometry.
+static void make_launch_args(const rr_read_params_t *p, const Geometry &g, const DeviceFacts &f,
+                             void *out_dev, void *scratch_dev, ReadArgs *a, Tables *tab)
+{
+    a->buf = (const char *)p->buf;
+    a->region_bytes = p->region_bytes;
+    a->reads = p->reads_per_warp;
+    a->first_read = p->first_read;
+    a->key_seed = sm64(p->seed);
+    a->n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
+    a->mode = p->mode;
+    a->ix.mode = p->index_mode;
+    a->ix.phase_shift = 0;
+    a->ix.sub_lines = 0;
+    if (p->index_mode == RR_INDEX_PHASED) {
+        while ((1u << a->ix.phase_shift) < p->phase_reads) ++a->ix.phase_shift;
+        const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
+        a->ix.sub_lines = sub > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sub;
+    }
+    a->n_warps = p->n_warps;
+    a->wps = g.wps;
+    a->wpc = g.wpc;
+    a->cps = g.cps;
+    a->nsm = (uint32_t)f.nsm;
+    a->n_groups = p->group_of_sm ? p->n_groups : 0;
+    a->pool_block = p->pool_block_reads ? p->pool_block_reads : 64u;
+    a->out = (uint2 *)out_dev;
+    a->scratch = (ScratchHeader *)scratch_dev;
+    std::memset(tab, 0, sizeof(*tab));
+    if (p->group_of_sm) {
+        std::memcpy(tab->group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
+        std::memcpy(tab->windows, p->windows, sizeof(rr_window_t) * p->n_groups);
+    }
+    if (p->mode == RR_MODE_POOLED)
+        std::memcpy(tab->warp_start, p->warp_start, sizeof(uint32_t) * (p->n_groups + 1));
+}
+
 static int32_t decode(const rr_read_params_t *p, const Geometry &g, const DeviceFacts &f,
                       const ScratchHeader &h, double seconds_event, rr_result_t *res)
 {
@@ -689,38 +726,8 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     }
 
     ReadArgs a;
-    a.buf = (const char *)p->buf;
-    a.region_bytes = p->region_bytes;
-    a.reads = p->reads_per_warp;
-    a.first_read = p->first_read;
-    a.key_seed = sm64(p->seed);
-    a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
-    a.mode = p->mode;
-    a.ix.mode = p->index_mode;
-    a.ix.phase_shift = 0;
-    a.ix.sub_lines = 0;
-    if (p->index_mode == RR_INDEX_PHASED) {
-        while ((1u << a.ix.phase_shift) < p->phase_reads) ++a.ix.phase_shift;
-        const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
-        a.ix.sub_lines = sub > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sub;
-    }
-    a.n_warps = p->n_warps;
-    a.wps = g.wps;
-    a.wpc = g.wpc;
-    a.cps = g.cps;
-    a.nsm = (uint32_t)f.nsm;
-    a.n_groups = p->group_of_sm ? p->n_groups : 0;
-    a.pool_block = p->pool_block_reads ? p->pool_block_reads : 64u;
-    a.out = (uint2 *)out_dev;
-    a.scratch = (ScratchHeader *)scratch_dev;
     Tables tab;
-    std::memset(&tab, 0, sizeof(tab));
-    if (p->group_of_sm) {
-        std::memcpy(tab.group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
-        std::memcpy(tab.windows, p->windows, sizeof(rr_window_t) * p->n_groups);
-    }
-    if (p->mode == RR_MODE_POOLED)
-        std::memcpy(tab.warp_start, p->warp_start, sizeof(uint32_t) * (p->n_groups + 1));
+    make_launch_args(p, g, f, out_dev, scratch_dev, &a, &tab);
 
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (res) {
@@ -1069,36 +1076,8 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
         if (rc != RR_OK) return rc;
     }
     ReadArgs a;
-    a.buf = (const char *)p->buf;
-    a.region_bytes = p->region_bytes;
-    a.reads = p->reads_per_warp;
-    a.first_read = p->first_read;
-    a.key_seed = sm64(p->seed);
-    a.n_lines = (uint32_t)(p->region_bytes / (128ull * p->words_per_lane));
-    a.mode = p->mode;
-    a.ix.mode = p->index_mode;
-    a.ix.phase_shift = 0;
-    a.ix.sub_lines = 0;
-    if (p->index_mode == RR_INDEX_PHASED) {
-        while ((1u << a.ix.phase_shift) < p->phase_reads) ++a.ix.phase_shift;
-        const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
-        a.ix.sub_lines = sub > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sub;
-    }
-    a.n_warps = p->n_warps;
-    a.wps = g.wps;
-    a.wpc = g.wpc;
-    a.cps = g.cps;
-    a.nsm = (uint32_t)f.nsm;
-    a.n_groups = p->group_of_sm ? p->n_groups : 0;
-    a.pool_block = 256u;
-    a.out = (uint2 *)out_dev;
-    a.scratch = (ScratchHeader *)scratch;
     Tables tab;
-    std::memset(&tab, 0, sizeof(tab));
-    if (p->group_of_sm) {
-        std::memcpy(tab.group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
-        std::memcpy(tab.windows, p->windows, sizeof(rr_window_t) * p->n_groups);
-    }
+    make_launch_args(p, g, f, out_dev, scratch, &a, &tab);
     // the array keeps the previous call's claims, counters and records: clear them
     RR_CUDA(cudaMemsetAsync(scratch, 0, kStaticUsedBytes, stream));
     if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
