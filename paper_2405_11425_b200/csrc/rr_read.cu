@@ -749,14 +749,15 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
         }                                      \
     } while (0)
 
-    RR_CUDA_C(cudaMemsetAsync(scratch_dev, 0, offsetof(ScratchHeader, probe), stream));
+    // claims, status, records -- and, in pooled mode, the work counters behind them
+    RR_CUDA_C(cudaMemsetAsync(scratch_dev, 0,
+                              p->mode == RR_MODE_POOLED ? sizeof(ScratchHeader)
+                                                        : offsetof(ScratchHeader, probe),
+                              stream));
     if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
         RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
-    if (p->mode == RR_MODE_POOLED) {  // work counters, and the checksums the atomics add into
-        RR_CUDA_C(cudaMemsetAsync(&((ScratchHeader *)scratch_dev)->pool_next, 0,
-                                  sizeof(unsigned long long) * RR_MAX_GROUPS, stream));
+    if (p->mode == RR_MODE_POOLED)  // the checksums the atomics add into
         RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)p->n_warps * sizeof(uint2), stream));
-    }
     if (res) RR_CUDA_C(cudaEventRecord(e0, stream));
     kernel<<<g.grid, g.block, smem, stream>>>(a, tab);
     RR_CUDA_C(cudaGetLastError());
