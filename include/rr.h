@@ -283,8 +283,8 @@ int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratc
  * (HOST) receives a GPC label per SM (numbered by smallest SM id), *n_gpcs their count.  No
  * timing is involved; every contention group found by rr_cluster on a probe matrix should lie
  * inside one of these GPCs (Section 2.2 found groups finer than GPCs).  nsm = the device's SM
- * count.  Synchronous; uses rr_scratch_bytes() of scratch.  RR_ERR_SM_UNCOVERED if some SM never
- * received a block.                                                                            */
+ * count.  Synchronous; uses rr_scratch_bytes() of scratch.  An SM that never hosted a block of
+ * any cluster stays a component of its own (it carries no placement information).             */
 int32_t rr_gpc_map(void *scratch_dev /*DEVICE*/, int32_t *gpc_of_sm_host /*HOST*/,
                    uint32_t *n_gpcs, uint32_t nsm, void *stream);
 

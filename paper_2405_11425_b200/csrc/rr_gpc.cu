@@ -47,7 +47,6 @@ extern "C" int32_t rr_gpc_map(void *scratch_dev, int32_t *gpc_of_sm_host, uint32
         return x;
     };
     std::vector<uint32_t> host(kGpcMaxBlocks);
-    std::vector<bool> seen(nsm, false);
     // cluster sizes 2..8 (portable), with a big and a small shared-memory footprint so that the
     // scheduler packs clusters differently; a few rounds each
     for (uint32_t csize = 2; csize <= 8; ++csize) {
@@ -79,19 +78,16 @@ extern "C" int32_t rr_gpc_map(void *scratch_dev, int32_t *gpc_of_sm_host, uint32
             for (uint32_t c = 0; c < blocks / csize; ++c) {
                 const uint32_t first = host[c * csize];
                 if (first >= nsm) continue;
-                seen[first] = true;
                 for (uint32_t k = 1; k < csize; ++k) {
                     const uint32_t s = host[c * csize + k];
                     if (s >= nsm) continue;
-                    seen[s] = true;
                     const uint32_t a = find(first), b = find(s);
                     if (a != b) parent[std::max(a, b)] = std::min(a, b);
                 }
             }
         }
     }
-    for (uint32_t s = 0; s < nsm; ++s)
-        if (!seen[s]) return RR_ERR_SM_UNCOVERED;
+    // an SM that never hosted a block of any cluster simply stays a component of its own
     // canonical labels: GPCs numbered by their smallest SM id
     std::vector<int32_t> label(nsm, -1);
     uint32_t G = 0;
