@@ -10,6 +10,7 @@
 // the slot of read t is folded into the checksums and immediately refilled with read t+U.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "rr_device.cuh"
@@ -1013,8 +1014,6 @@ extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint6
 // For callers that cannot obtain device memory of their own (see rr.h).  The scratch lives in a
 // file-scope device array; in host code its name is only a handle, so the device address is
 // fetched once per device with cudaGetSymbolAddress and cached here.
-#include <mutex>
-
 namespace rr {
 
 constexpr uint32_t kStaticMaxSm = RR_STATIC_MAX_SM;
