@@ -57,6 +57,41 @@ def aggregate_throughput(local_bytes: float, local_seconds: float, group=None) -
     return float(b.item()), float(s.item())
 
 
+def save_calibration(path, uuid: str, groups: "Groups", reach: "Reach | None" = None,
+                     weights=None) -> None:
+    """Writes what was measured on one card (SM groups, reach, capacity weights) as JSON, keyed by
+    the GPU's UUID: the layout is a property of the card (Section 1.1), so it can be reused."""
+    import json
+    doc = {"uuid": uuid, "n_groups": int(groups.n_groups), "confidence": float(groups.confidence),
+           "group_of_sm": [int(g) for g in groups.group_of_sm],
+           "reach": None if reach is None else {"cliff": bool(reach.cliff),
+                                                "plateau_gbps": float(reach.plateau_gbps),
+                                                "reach_bytes": int(reach.reach_bytes)},
+           "weights": None if weights is None else [int(w) for w in weights]}
+    with open(path, "w") as f:
+        json.dump(doc, f)
+
+
+def load_calibration(path, uuid: str, nsm: int):
+    """Reads a calibration written by save_calibration; refuses one taken on another card or with
+    another SM count.  Returns (Groups, Reach or None, weights or None)."""
+    import json
+    with open(path) as f:
+        doc = json.load(f)
+    if doc.get("uuid") != uuid:
+        raise ValueError(f"calibration belongs to GPU {doc.get('uuid')}, this is {uuid}")
+    g = np.asarray(doc["group_of_sm"], dtype=np.uint16)
+    if g.shape != (nsm,) or int(g.max()) + 1 != doc["n_groups"]:
+        raise ValueError("calibration does not describe this SM count")
+    groups = Groups(g, int(doc["n_groups"]), float(doc["confidence"]), None, 1.0, 0.0,
+                    np.bincount(g, minlength=doc["n_groups"]).tolist())
+    r = doc.get("reach")
+    reach = None if r is None else Reach(bool(r["cliff"]), float(r["plateau_gbps"]),
+                                         int(r["reach_bytes"]), [])
+    w = doc.get("weights")
+    return groups, reach, None if w is None else np.asarray(w, dtype=np.uint32)
+
+
 def rebalanced_weights(work, finish_ns, scale: int = 1_000_000) -> np.ndarray:
     """New integer group weights from one balanced-run observation: a group that did `work`
     units and finished after `finish_ns` has shown a rate work/finish; weights are those rates,

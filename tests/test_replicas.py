@@ -10,8 +10,9 @@ import torch.multiprocessing as mp
 
 import numpy as np
 
-from paper_2405_11425_b200.pipeline import (aggregate_throughput, finish_spread,
-                                             rebalanced_weights)
+from paper_2405_11425_b200.pipeline import (Groups, Reach, aggregate_throughput, finish_spread,
+                                             load_calibration, rebalanced_weights,
+                                             save_calibration)
 
 
 def _free_port():
@@ -66,3 +67,17 @@ def test_rebalancing_moves_work_towards_groups_that_finished_early():
     assert finish_spread([1000.0, 980.0, 0.0]) == pytest.approx(0.02)
     with pytest.raises(ValueError):
         rebalanced_weights([1, 1], [0.0, 0.0])
+
+
+def test_calibration_round_trip_is_bound_to_the_card(tmp_path):
+    g = Groups(np.array([0, 0, 1, 1, 2, 2], np.uint16), 3, 47.0)
+    r = Reach(True, 4600.0, 70 << 30, [(1 << 30, 5400.0)])
+    path = tmp_path / "card.json"
+    save_calibration(path, "abc123", g, r, weights=[5, 6, 7])
+    g2, r2, w2 = load_calibration(path, "abc123", 6)
+    assert np.array_equal(g2.group_of_sm, g.group_of_sm) and g2.n_groups == 3 and g2.sizes == [2, 2, 2]
+    assert r2.cliff and r2.reach_bytes == 70 << 30 and list(w2) == [5, 6, 7]
+    with pytest.raises(ValueError):
+        load_calibration(path, "another-card", 6)
+    with pytest.raises(ValueError):
+        load_calibration(path, "abc123", 8)
