@@ -62,9 +62,9 @@ def _load():
         lib.orc_warp_checksum.restype = None
         lib.orc_warp_checksum.argtypes = [u32, u64, u64, u64, u64, u64, u32, u64, u64, p, p]
         lib.orc_line_phased.restype = u64
-        lib.orc_line_phased.argtypes = [u64, u64, u64, u64, u64, u64, u64]
+        lib.orc_line_phased.argtypes = [u64, u64, u64, u64, u64, u64, u64, u64]
         lib.orc_warp_checksum_phased.restype = None
-        lib.orc_warp_checksum_phased.argtypes = [u64, u64, u64, u64, u32, u64, u64, u64, u64, p, p]
+        lib.orc_warp_checksum_phased.argtypes = [u64, u64, u64, u64, u32, u64, u64, u64, u64, u64, p, p]
         lib.orc_read_per_sm_phased.restype = i32
         lib.orc_read_per_sm_phased.argtypes = [u64, u32, u32, u32, u64, u64, u64, p, p, p, u32, u64,
                                                u64, p]
@@ -182,16 +182,21 @@ def read_per_sm(region_bytes: int, W: int, nsm: int, wps: int, reads: int, seed:
 
 
 def line_phased(seed: int, v: int, i: int, base: int, n: int, phase_reads: int,
-                sub_lines: int) -> int:
-    return int(_load().orc_line_phased(seed, v, i, base, n, phase_reads, sub_lines))
+                sub_lines: int, stagger: int = 0) -> int:
+    return int(_load().orc_line_phased(seed, v, i, base, n, phase_reads, sub_lines, stagger))
+
+
+def stagger_of_sm(sm: int, nsm: int, n: int, sub_lines: int) -> int:
+    """Shift of SM `sm`'s phase cycle in per-SM mode: floor(sm * Q / nsm), Q = ceil(n/sub_lines)."""
+    return sm * (-(-n // sub_lines)) // nsm
 
 
 def warp_checksum_phased(seed: int, v: int, first_read: int, reads: int, W: int, base: int, n: int,
-                         phase_reads: int, sub_lines: int):
+                         phase_reads: int, sub_lines: int, stagger: int = 0):
     x = ctypes.c_uint32()
     s = ctypes.c_uint32()
     _load().orc_warp_checksum_phased(seed, v, first_read, reads, W, base, n, phase_reads, sub_lines,
-                                     ctypes.byref(x), ctypes.byref(s))
+                                     stagger, ctypes.byref(x), ctypes.byref(s))
     return int(x.value), int(s.value)
 
 

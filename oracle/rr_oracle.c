@@ -131,23 +131,27 @@ void orc_warp_checksum(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t 
  * in phases of phase_reads reads, phase p = floor(i / phase_reads) of a warp's stream
  * (i = absolute read counter) draws uniformly inside sub-window p mod Q.  Over Q
  * phases every line of the window is equally likely; at any moment a warp is held to
- * n/Q lines.  With sub_lines >= n this is the plain random mode.                    */
+ * n/Q lines.  With sub_lines >= n this is the plain random mode.
+ * stagger shifts the cycle: sub-window (p + stagger) mod Q.  In per-SM mode SM s of nsm
+ * uses stagger = floor(s * Q / nsm), so that SMs sharing one window (all of memory, say)
+ * are spread over its sub-windows instead of crowding into one.                      */
 uint64_t orc_line_phased(uint64_t seed, uint64_t v, uint64_t i, uint64_t base, uint64_t n,
-                         uint64_t phase_reads, uint64_t sub_lines)
+                         uint64_t phase_reads, uint64_t sub_lines, uint64_t stagger)
 {
     uint64_t Q = (n + sub_lines - 1) / sub_lines;
-    uint64_t q = (i / phase_reads) % Q;
+    uint64_t q = (i / phase_reads + stagger) % Q;
     uint64_t lo = n * q / Q, hi = n * (q + 1) / Q; /* n < 2^32, Q <= n: fits 64 bits */
     return base + lo + orc_draw(seed, v, i) % (hi - lo);
 }
 
 void orc_warp_checksum_phased(uint64_t seed, uint64_t v, uint64_t first_read, uint64_t reads,
                               uint32_t W, uint64_t base, uint64_t n, uint64_t phase_reads,
-                              uint64_t sub_lines, uint32_t *X, uint32_t *S)
+                              uint64_t sub_lines, uint64_t stagger, uint32_t *X, uint32_t *S)
 {
     uint32_t x = 0, s = 0;
     for (uint64_t t = 0; t < reads; ++t) {
-        uint64_t line = orc_line_phased(seed, v, first_read + t, base, n, phase_reads, sub_lines);
+        uint64_t line = orc_line_phased(seed, v, first_read + t, base, n, phase_reads, sub_lines,
+                                        stagger);
         for (uint32_t lane = 0; lane < 32; ++lane)
             for (uint32_t w = 0; w < W; ++w) {
                 uint32_t word = orc_word(line * 32u * W + (uint64_t)lane * W + w);
@@ -195,8 +199,10 @@ int32_t orc_read_per_sm_phased(uint64_t region_bytes, uint32_t W, uint32_t nsm, 
             base = win_base[group_of_sm[sm]];
             n = win_n[group_of_sm[sm]];
         }
+        uint64_t Q = (n + sub - 1) / sub;
+        uint64_t stagger = (uint64_t)sm * Q / nsm;
         orc_warp_checksum_phased(seed, (uint64_t)v, first_read, reads, W, base, n, phase_reads, sub,
-                                 &out[2 * v], &out[2 * v + 1]);
+                                 stagger, &out[2 * v], &out[2 * v + 1]);
     }
     return ORC_OK;
 }

@@ -55,12 +55,13 @@ def test_checksums_follow_the_lines():
             continue
         base, n = map(int, windows[groups[sm]])
         x = s = 0
+        st = oracle.stagger_of_sm(sm, 4, n, 1000)
         for i in range(64, 164):
-            w = oracle.fill(oracle.line_phased(5, v, i, base, n, 32, 1000) * 32, 32)
+            w = oracle.fill(oracle.line_phased(5, v, i, base, n, 32, 1000, st) * 32, 32)
             x ^= int(np.bitwise_xor.reduce(w))
             s = (s + int(w.astype(np.uint64).sum())) & 0xFFFFFFFF
         assert tuple(out[v]) == (x, s)
-        assert tuple(out[v]) == oracle.warp_checksum_phased(5, v, 64, 100, 1, base, n, 32, 1000)
+        assert tuple(out[v]) == oracle.warp_checksum_phased(5, v, 64, 100, 1, base, n, 32, 1000, st)
 
 
 def test_a_full_cycle_covers_the_window_uniformly():
@@ -77,3 +78,19 @@ def test_errors():
         oracle.read_per_sm_phased(1 << 20, 1, 2, 2, 4, 1, phase_reads=0, phase_window_bytes=1 << 16)
     with pytest.raises(oracle.OracleError):
         oracle.read_per_sm_phased(1 << 20, 1, 2, 2, 4, 1, phase_reads=32, phase_window_bytes=64)
+
+
+def test_stagger_spreads_sms_that_share_one_window():
+    # 8 SMs, one window cut into 4 sub-windows: in any phase the SMs sit two per sub-window,
+    # and each SM still cycles through all four
+    n, B, sub, nsm = 4000, 32, 1000, 8
+    for phase in range(6):
+        seen = []
+        for sm in range(nsm):
+            st = oracle.stagger_of_sm(sm, nsm, n, sub)
+            assert st == sm * 4 // nsm
+            seen.append(oracle.line_phased(1, sm * 2, phase * B, 0, n, B, sub, st) * 4 // n)
+        assert sorted(seen) == [0, 0, 1, 1, 2, 2, 3, 3]
+    cycle = [oracle.line_phased(1, 6, p * B, 0, n, B, sub, oracle.stagger_of_sm(3, nsm, n, sub)) * 4 // n
+             for p in range(4)]
+    assert sorted(cycle) == [0, 1, 2, 3]
