@@ -28,7 +28,8 @@
  *                  (RR_INDEX_PHASED: the window is cut into Q = ceil(n / sub) sub-windows
  *                  [floor(n q / Q), floor(n (q+1) / Q)), sub = phase_window_bytes / (128 W);
  *                  read i belongs to phase p = floor(i / phase_reads) and draws
- *                  base + lo_q + (r mod (hi_q - lo_q)) with q = p mod Q)
+ *                  base + lo_q + (r mod (hi_q - lo_q)) with q = (p + stagger) mod Q, where
+ *                  stagger = floor(smid * Q / nsm) in RR_MODE_PER_SM and 0 otherwise)
  *   checksum     = {X, S}: X = xor, S = sum mod 2^32 of every 32-bit word the warp read
  */
 #ifndef RR_H_
@@ -135,6 +136,8 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   wants each warp held to a smaller region; here that region also moves, so that an SM whose
  *   own translation cache is smaller than its share of memory works through its window one
  *   sub-window at a time while a whole cycle of phases still covers the window uniformly.
+ *   SMs that share a window (the whole region when group_of_sm is NULL) start their cycles at
+ *   staggered sub-windows, so the region can also be read from every SM with no partition.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered

@@ -29,6 +29,7 @@ struct IndexSpec {
     uint32_t mode;         // RR_INDEX_*
     uint32_t phase_shift;  // PHASED: log2(reads per phase)
     uint32_t sub_lines;    // PHASED: largest sub-window, in lines
+    uint32_t sm, nsm;      // PHASED, per-SM mode: this SM of nsm (nsm = 0: no stagger)
 };
 
 // The window a batch of 32 reads draws from: the warp's whole window, or (PHASED) the
@@ -37,7 +38,7 @@ struct LineSource {
     uint32_t base;
     Divisor div;
     uint32_t win_base, win_n;
-    uint64_t n_sub, phase;
+    uint64_t n_sub, phase, stagger;
     __device__ __forceinline__ void init(uint32_t b, uint32_t n, const IndexSpec &ix)
     {
         win_base = base = b;
@@ -45,6 +46,8 @@ struct LineSource {
         div = make_divisor(n);
         phase = ~0ull;
         n_sub = ix.mode == RR_INDEX_PHASED ? ((uint64_t)n + ix.sub_lines - 1) / ix.sub_lines : 1;
+        // SMs that share a window start their cycles at different sub-windows
+        stagger = (ix.mode == RR_INDEX_PHASED && ix.nsm) ? (uint64_t)ix.sm * n_sub / ix.nsm : 0;
     }
     // i0 = absolute index of the first read of a batch; all 32 reads of a batch share a phase
     // because phases are multiples of 32 reads and streams start at multiples of 32
@@ -54,7 +57,7 @@ struct LineSource {
         const uint64_t p = i0 >> ix.phase_shift;
         if (p == phase) return;
         phase = p;
-        const uint64_t q = p % n_sub;
+        const uint64_t q = (p + stagger) % n_sub;
         const uint64_t lo = (uint64_t)win_n * q / n_sub, hi = (uint64_t)win_n * (q + 1) / n_sub;
         base = win_base + (uint32_t)lo;
         div = make_divisor((uint32_t)(hi - lo));
@@ -368,8 +371,11 @@ __global__ void __launch_bounds__(1024, 1)
         const uint64_t v = (uint64_t)sm * a.wps + slot * a.wpc + warp;
         const uint64_t V = (uint64_t)a.nsm * a.wps;
         uint32_t X, S;
-        warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v, V,
-                                  a.first_read, a.reads, base, n, lane, X, S, &sc->violations);
+        IndexSpec ix = a.ix;
+        ix.sm = sm;
+        ix.nsm = a.nsm;
+        warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), ix, v, V, a.first_read,
+                              a.reads, base, n, lane, X, S, &sc->violations);
         if (lane == 0) a.out[v] = make_uint2(X, S);
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -439,7 +445,7 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     const uint64_t v = (uint64_t)sm * a.wps + warp;
     uint32_t X, S;
     warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
-                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u}, v,
+                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u}, v,
                                        (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
                                        a.n_lines, lane, X, S, nullptr);
     if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
@@ -639,6 +645,8 @@ static void make_launch_args(const rr_read_params_t *p, const Geometry &g, const
     a->ix.mode = p->index_mode;
     a->ix.phase_shift = 0;
     a->ix.sub_lines = 0;
+    a->ix.sm = 0;
+    a->ix.nsm = 0;  // set by the block in per-SM mode
     if (p->index_mode == RR_INDEX_PHASED) {
         while ((1u << a->ix.phase_shift) < p->phase_reads) ++a->ix.phase_shift;
         const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);

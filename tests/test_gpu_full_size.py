@@ -256,5 +256,25 @@ def test_moving_windows_over_the_whole_buffer_sampled(ses):
     got = ses.checksums(ses.nsm * WPS)
     for v in _sample(ses.nsm * WPS):
         base, n = map(int, win[owners[v // WPS]])
+        st = oracle.stagger_of_sm(v // WPS, ses.nsm, n, sub_bytes // 128)
         assert tuple(got[v]) == oracle.warp_checksum_phased(rr_inputs.CFG4_SEED, v, first, reads, 1,
-                                                            base, n, 1024, sub_bytes // 128), v
+                                                            base, n, 1024, sub_bytes // 128, st), v
+
+
+def test_moving_window_over_all_of_memory_from_every_sm_sampled(ses):
+    # no partition at all: every SM's window is the whole buffer, cut into 128 MiB sub-windows,
+    # SMs staggered over them
+    region = ses.region_bytes
+    reads = 256 * 64
+    sub_bytes = 128 << 20
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=reads, seed=7,
+                   variant=rr.RR_VARIANT_PACKED, unroll=2, index_mode=rr.RR_INDEX_PHASED,
+                   phase_reads=1024, phase_window_bytes=sub_bytes)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == ses.nsm
+    got = ses.checksums(ses.nsm * WPS)
+    L = region // 128
+    for v in _sample(ses.nsm * WPS):
+        st = oracle.stagger_of_sm(v // WPS, ses.nsm, L, sub_bytes // 128)
+        assert tuple(got[v]) == oracle.warp_checksum_phased(7, v, 0, reads, 1, 0, L, 1024,
+                                                            sub_bytes // 128, st), v

@@ -378,6 +378,15 @@ def test_phased_index_mode_matches_oracle(dev, W, variant):
                       seed=3, variant=variant, index_mode=rr.RR_INDEX_PHASED, phase_reads=32,
                       phase_window_bytes=64 << 20)
     rr.rr_random_read(p, out, dev.scratch)
-    expect = oracle.read_per_sm_phased(region, W, 2, 32, 200, 3, 32, 64 << 20,
-                                       group_of_sm=np.zeros(2, np.uint16), windows=[[0, L]])
-    assert np.array_equal(_np(out), expect)
+    got = _np(out)
+    sub = (64 << 20) // (128 * W)
+    for v in range(64):                              # logical warps: no SM, so no stagger
+        assert tuple(got[v]) == oracle.warp_checksum_phased(3, v, 0, 200, W, 0, L, 32, sub, 0)
+    # every SM on the whole region: the SMs start their cycles at staggered sub-windows
+    out = _out(dev, dev.nsm * 4)
+    p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=4, reads_per_warp=160, seed=3,
+                      variant=variant, index_mode=rr.RR_INDEX_PHASED, phase_reads=32,
+                      phase_window_bytes=8 << 20)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_per_sm_phased(region, W, dev.nsm, 4, 160, 3, 32,
+                                                              8 << 20))
