@@ -265,6 +265,21 @@ def run_gpu(args):
     ev1.record()
     torch.cuda.synchronize()
     moving_gbps = rr.rr_read_report(mv, ses.scratch).bytes * 100 / ev0.elapsed_time(ev1) * 1e-6
+    # and with no partition at all: every SM's window is the whole buffer, 128 MiB sub-windows,
+    # the SMs' cycles staggered
+    mv_all = ses.params(N, W=1, warps_per_sm=WARPS_PER_SM,
+                        reads_per_warp=READS_PER_ITER * ITERS_PER_STEP, seed=SEED,
+                        variant=VARIANT_PACKED, unroll=UNROLL, index_mode=rr.RR_INDEX_PHASED,
+                        phase_reads=1024, phase_window_bytes=128 << 20)
+    for _ in range(SETTLE_LAUNCHES):
+        rr.rr_random_read(mv_all, ses.out, ses.scratch, timed=False)
+    ev0.record()
+    for _ in range(100):
+        rr.rr_random_read(mv_all, ses.out, ses.scratch, timed=False)
+    ev1.record()
+    torch.cuda.synchronize()
+    moving_all_gbps = (rr.rr_read_report(mv_all, ses.scratch).bytes * 100
+                       / ev0.elapsed_time(ev1) * 1e-6)
     t_cal = time.time() - t_cal
 
     # ---- timed region: device-resident, asynchronous launches -------------------------------
@@ -404,7 +419,11 @@ def run_gpu(args):
                 "moving_windows": {"gbps_sustained": moving_gbps, "phase_reads": 1024,
                                    "sub_window_mib": mv_sub / (1 << 20), "sub_windows": 8,
                                    "note": "same per-SM slices, equal work per SM, each SM held "
-                                           "to one eighth of its slice at a time"},
+                                           "to one eighth of its slice at a time",
+                                   "no_partition_gbps_sustained": moving_all_gbps,
+                                   "no_partition_note": "every SM's window is the whole buffer, "
+                                                        "128 MiB sub-windows, 1024 reads per "
+                                                        "phase, SM cycles staggered"},
                 "equal_work_per_sm": {"window": headline, "window_gib": S / GiB,
                                       "coverage": coverage,
                                       "gbps": window_sweep[headline]["gbps"]},

@@ -188,6 +188,26 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                            "phase_reads": B,
                            "sustained_gbps": rep.bytes * n / e0.elapsed_time(e1) * 1e-6})
     R["moving_windows"] = moving
+    # no partition: every SM's window is the whole buffer, SM cycles staggered
+    moving_all = []
+    for sub_mib in (64, 128, 256, 512):
+        for B in (1024, 4096):
+            p = ses.params(N, seed=23, reads_per_warp=reads, variant=rr.RR_VARIANT_PACKED, unroll=2,
+                           index_mode=rr.RR_INDEX_PHASED, phase_reads=B,
+                           phase_window_bytes=sub_mib * MiB)
+            n = 30 if quick else 200
+            for _ in range(10 if quick else 100):
+                rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                rr.rr_random_read(p, ses.out, ses.scratch, timed=False)
+            e1.record()
+            torch.cuda.synchronize()
+            rep = rr.rr_read_report(p, ses.scratch)
+            moving_all.append({"sub_window_mib": sub_mib, "phase_reads": B,
+                               "sustained_gbps": rep.bytes * n / e0.elapsed_time(e1) * 1e-6})
+    R["moving_windows_no_partition"] = moving_all
 
     # work in proportion to group capacity (pooled mode), balanced under sustained load
     balanced = {}
@@ -294,6 +314,11 @@ def markdown(R: dict) -> str:
     for r in R.get("moving_windows", []):
         L.append(f"| {r['sub_windows']} | {r['sub_window_mib']:.0f} | {r['phase_reads']} | "
                  f"{r['sustained_gbps']:.0f} |")
+    L.append("")
+    L += ["## Moving windows with no partition: every SM's window is the whole buffer", "",
+          "| sub-window MiB | reads per phase | GB/s |", "|---|---|---|"]
+    for r in R.get("moving_windows_no_partition", []):
+        L.append(f"| {r['sub_window_mib']} | {r['phase_reads']} | {r['sustained_gbps']:.0f} |")
     L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]
