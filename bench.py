@@ -249,9 +249,16 @@ def run_gpu(args):
     t_bal = time.time() - t_bal
 
     # the same slices with windows that move (phased index): every SM works through its slice in
-    # eight sub-windows, one per 1024 reads, so that its own translation cache holds the live part
+    # sub-windows, one per 1024 reads, sized so that its own translation cache holds the live part
+    sm_reach, sm_reach_points = ses.measure_sm_reach()
     mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
-    mv_sub = (int(mv_windows[:, 1].max()) * 128 + 7) // 8
+    slice_bytes = int(mv_windows[:, 1].max()) * 128
+    # two phases can be live at once and the cache should hold both with room to spare:
+    # sub-windows of at most a quarter of the SM's reach, a power-of-two number per slice
+    mv_parts = 1
+    while slice_bytes / mv_parts > sm_reach / 4 and mv_parts < 64:
+        mv_parts *= 2
+    mv_sub = (slice_bytes + mv_parts - 1) // mv_parts
     mv = ses.params(N, W=1, warps_per_sm=WARPS_PER_SM, reads_per_warp=READS_PER_ITER * ITERS_PER_STEP,
                     seed=SEED, group_of_sm=owners.group_of_sm, windows=mv_windows,
                     variant=VARIANT_PACKED, unroll=UNROLL, index_mode=rr.RR_INDEX_PHASED,
@@ -265,12 +272,12 @@ def run_gpu(args):
     ev1.record()
     torch.cuda.synchronize()
     moving_gbps = rr.rr_read_report(mv, ses.scratch).bytes * 100 / ev0.elapsed_time(ev1) * 1e-6
-    # and with no partition at all: every SM's window is the whole buffer, 128 MiB sub-windows,
-    # the SMs' cycles staggered
+    # and with no partition at all: every SM's window is the whole buffer, the same sub-window
+    # size, the SMs' cycles staggered
     mv_all = ses.params(N, W=1, warps_per_sm=WARPS_PER_SM,
                         reads_per_warp=READS_PER_ITER * ITERS_PER_STEP, seed=SEED,
                         variant=VARIANT_PACKED, unroll=UNROLL, index_mode=rr.RR_INDEX_PHASED,
-                        phase_reads=1024, phase_window_bytes=128 << 20)
+                        phase_reads=1024, phase_window_bytes=mv_sub)
     for _ in range(SETTLE_LAUNCHES):
         rr.rr_random_read(mv_all, ses.out, ses.scratch, timed=False)
     ev0.record()
@@ -416,13 +423,15 @@ def run_gpu(args):
                             "warps_per_window_min_max": [
                                 int(np.diff(warp_start.astype(np.int64)).min()),
                                 int(np.diff(warp_start.astype(np.int64)).max())]},
+                "sm_reach": {"reach_mib": sm_reach / (1 << 20),
+                             "sweep": [[b / (1 << 20), g] for b, g in sm_reach_points]},
                 "moving_windows": {"gbps_sustained": moving_gbps, "phase_reads": 1024,
-                                   "sub_window_mib": mv_sub / (1 << 20), "sub_windows": 8,
+                                   "sub_window_mib": mv_sub / (1 << 20), "sub_windows": mv_parts,
                                    "note": "same per-SM slices, equal work per SM, each SM held "
-                                           "to one eighth of its slice at a time",
+                                           "to one sub-window of its slice at a time",
                                    "no_partition_gbps_sustained": moving_all_gbps,
                                    "no_partition_note": "every SM's window is the whole buffer, "
-                                                        "128 MiB sub-windows, 1024 reads per "
+                                                        "same sub-window size, 1024 reads per "
                                                         "phase, SM cycles staggered"},
                 "equal_work_per_sm": {"window": headline, "window_gib": S / GiB,
                                       "coverage": coverage,

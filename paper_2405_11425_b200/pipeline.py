@@ -205,6 +205,30 @@ class Session:
             cliff, plateau, reach = rr.rr_reach([p[0] for p in pts], [p[1] for p in pts])
         return Reach(cliff, plateau, reach, pts)
 
+    def measure_sm_reach(self, sizes_mib=(32, 64, 128, 256, 384, 512, 768, 1024), *,
+                         keep: float = 0.97, seed: int = 23, reads_per_warp: int = 256 * 16):
+        """How large a window can one SM read at random before its own translation cache stops
+        covering it?  Every SM gets a window of the given size (windows spread over the buffer,
+        equal work); the answer is the largest size whose rate stays within `keep` of the rate
+        at the smallest sizes.  Returns (reach_bytes, [(size_bytes, GB/s)])."""
+        ids = np.arange(self.nsm, dtype=np.uint16)
+        stride = (self.region_bytes // 128) // self.nsm
+        pts = []
+        for mib in sizes_mib:
+            n = min((mib << 20) // 128, stride)
+            win = np.array([[k * stride, n] for k in range(self.nsm)], np.uint32)
+            g, _ = self.read(self.region_bytes, seed=seed, reads_per_warp=reads_per_warp,
+                             group_of_sm=ids, windows=win)
+            pts.append((int(n) * 128, g))
+        top = sorted(p[1] for p in pts[:3])[1]
+        reach = pts[0][0]
+        for size, g in pts:
+            if g >= keep * top:
+                reach = size
+            else:
+                break
+        return reach, pts
+
     # -- groups -----------------------------------------------------------------------------
     def discover_groups(self, *, probe_region_bytes=None, total_reads: int = 1 << 18,
                         warps_per_sm: int = 32, seed: int = 5, repeats: int = 3,
