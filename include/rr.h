@@ -73,9 +73,29 @@ extern "C" {
 #define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
 #define RR_VARIANT_PACKED 2u      /* every lane loads 16 bytes: one warp load covers 4/W lines  */
                                   /* (same lines and words; fewer instructions per line)        */
+#define RR_VARIANT_L2_128 3u      /* RR_VARIANT_LDG with the .L2::128B prefetch qualifier       */
+#define RR_VARIANT_L2_256 4u      /* RR_VARIANT_LDG with the .L2::256B prefetch qualifier       */
+#define RR_VARIANT_BULK 5u        /* one cp.async.bulk per line into a ring in shared memory,   */
+                                  /* completion on an mbarrier, lanes fold from shared memory   */
 
 const char *rr_strerror(int32_t code);
 const char *rr_last_cuda_error(void);
+
+/* ---- host-side bookkeeping the library keeps ----------------------------------------------
+ * Three small caches live in the library for the life of the process, none of them on the
+ * device: the attributes of each device (asked once), the launch configuration of each
+ * (device, kernel, block size, blocks per SM) -- the dynamic shared-memory request that keeps one
+ * block per SM, found by an occupancy search -- and two timing events per host thread and
+ * device.  A repeated call therefore makes no attribute, occupancy or event-creation call.
+ * rr_host_counters reports how often each of those runtime calls was really made (HOST struct);
+ * it exists so that a test can see the caches work.                                            */
+typedef struct {
+    uint64_t occupancy_queries;   /* cudaOccupancyMaxActiveBlocksPerMultiprocessor calls         */
+    uint64_t attribute_sets;      /* cudaFuncSetAttribute calls                                  */
+    uint64_t event_creates;       /* cudaEventCreate calls                                       */
+    uint64_t device_fact_queries; /* rounds of cudaDeviceGetAttribute queries                    */
+} rr_host_counters_t;
+int32_t rr_host_counters(rr_host_counters_t *out /*HOST*/);
 
 /* ---- device facts ------------------------------------------------------------------------
  * Paper, Section 1.1: the %smid / %nsmid registers are the only layout facts a program gets.

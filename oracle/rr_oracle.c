@@ -390,12 +390,15 @@ int32_t orc_read_pooled(uint64_t region_bytes, uint32_t W, uint32_t n_groups,
         if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
     }
     uint64_t V = warp_start[n_groups];
-    for (uint32_t g = 0; g < n_groups; ++g) {
-        int64_t lo = warp_start[g], hi = warp_start[g + 1];
-#pragma omp parallel for schedule(dynamic, 16)
-        for (int64_t v = lo; v < hi; ++v)
-            orc_warp_checksum(ORC_INDEX_RANDOM, seed, (uint64_t)v, V, first_read, reads, W,
-                              win_base[g], win_n[g], &out[2 * v], &out[2 * v + 1]);
+    int64_t nw = (int64_t)V;
+    /* one loop over all warps (they are independent), so that every host core has work
+     * whatever the number of groups; the owner of warp v is looked up by its range */
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t g = 0;
+        while (!((uint64_t)v >= warp_start[g] && (uint64_t)v < warp_start[g + 1])) ++g;
+        orc_warp_checksum(ORC_INDEX_RANDOM, seed, (uint64_t)v, V, first_read, reads, W,
+                          win_base[g], win_n[g], &out[2 * v], &out[2 * v + 1]);
     }
     return ORC_OK;
 }

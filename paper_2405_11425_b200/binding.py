@@ -24,13 +24,14 @@ RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0x
 RR_MODE_LOGICAL, RR_MODE_PER_SM, RR_MODE_POOLED = 0, 1, 2
 RR_INDEX_RANDOM, RR_INDEX_STRIDE, RR_INDEX_PHASED = 0, 1, 2
 RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED, RR_VARIANT_PACKED = 0, 1, 2
+RR_VARIANT_L2_128, RR_VARIANT_L2_256, RR_VARIANT_BULK = 3, 4, 5
 
 EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
     "rr_random_read", "rr_read_report", "rr_probe_pair", "rr_probe_matrix_scratch_bytes",
     "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach", "rr_random_read_static",
     "rr_gpc_map", "rr_make_weighted_windows",
-    "rr_read_block_times",
+    "rr_read_block_times", "rr_host_counters",
 )
 
 
@@ -148,6 +149,8 @@ def _load():
     lib.rr_make_weighted_windows.argtypes = [u64, u32, u32, p, u32, u64, p, p]
     lib.rr_reach.restype = i32
     lib.rr_reach.argtypes = [p, p, u32, p, p]
+    lib.rr_host_counters.restype = i32
+    lib.rr_host_counters.argtypes = [p]
     _lib = lib
     return lib
 
@@ -186,6 +189,14 @@ def rr_device_info() -> dict:
     out["name"] = info.name.decode()
     out["uuid"] = info.uuid.decode()
     return out
+
+
+def rr_host_counters() -> dict:
+    """How often the library really asked the runtime for occupancy, attributes, events, facts."""
+    c = (ctypes.c_uint64 * 4)()
+    _check(_load().rr_host_counters(c), "rr_host_counters")
+    return dict(zip(("occupancy_queries", "attribute_sets", "event_creates",
+                     "device_fact_queries"), (int(x) for x in c)))
 
 
 def rr_scratch_bytes() -> int:

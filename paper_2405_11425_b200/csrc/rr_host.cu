@@ -1,7 +1,9 @@
 // Host-only parts of librr: status strings, device facts, the window policy and the reach rule.
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "rr_device.cuh"
@@ -18,16 +20,36 @@ void set_cuda_error(cudaError_t e, const char *what)
     cudaGetLastError();  // clear the sticky-less error state
 }
 
+// Facts of each device are asked of the runtime once and kept: they cannot change while the
+// process lives, and six attribute queries per launch are visible next to a 2 ms kernel.
+static std::mutex g_facts_mutex;
+static DeviceFacts g_facts[64];
+static bool g_facts_known[64];
+static std::atomic<uint64_t> g_n_fact_queries{0};
+
+uint64_t device_fact_queries() { return g_n_fact_queries.load(); }
+
 int32_t device_facts(DeviceFacts *out)
 {
-    RR_CUDA(cudaGetDevice(&out->device));
-    RR_CUDA(cudaDeviceGetAttribute(&out->nsm, cudaDevAttrMultiProcessorCount, out->device));
-    RR_CUDA(cudaDeviceGetAttribute(&out->cc_major, cudaDevAttrComputeCapabilityMajor, out->device));
-    RR_CUDA(cudaDeviceGetAttribute(&out->cc_minor, cudaDevAttrComputeCapabilityMinor, out->device));
-    RR_CUDA(cudaDeviceGetAttribute(&out->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor,
-                                   out->device));
-    RR_CUDA(cudaDeviceGetAttribute(&out->smem_per_block_optin,
-                                   cudaDevAttrMaxSharedMemoryPerBlockOptin, out->device));
+    int dev = 0;
+    RR_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_facts_mutex);
+    if (!g_facts_known[dev]) {
+        DeviceFacts f;
+        f.device = dev;
+        g_n_fact_queries.fetch_add(1);
+        RR_CUDA(cudaDeviceGetAttribute(&f.nsm, cudaDevAttrMultiProcessorCount, dev));
+        RR_CUDA(cudaDeviceGetAttribute(&f.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+        RR_CUDA(cudaDeviceGetAttribute(&f.cc_minor, cudaDevAttrComputeCapabilityMinor, dev));
+        RR_CUDA(cudaDeviceGetAttribute(&f.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor,
+                                       dev));
+        RR_CUDA(cudaDeviceGetAttribute(&f.smem_per_block_optin,
+                                       cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        g_facts[dev] = f;
+        g_facts_known[dev] = true;
+    }
+    *out = g_facts[dev];
     if (out->cc_major != 10) {
         std::snprintf(g_cuda_error, sizeof(g_cuda_error),
                       "device has compute capability %d.%d; this library holds sm_100a code only",

@@ -60,5 +60,6 @@ struct DeviceFacts {
     int smem_per_block_optin;
 };
 int32_t device_facts(DeviceFacts *out);
+uint64_t device_fact_queries();  // how often the runtime was really asked
 
 }  // namespace rr

@@ -9,6 +9,7 @@
 // vector load fetches the lane's W words.  U loads per warp stay in flight in a register ring:
 // the slot of read t is folded into the checksums and immediately refilled with read t+U.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -81,9 +82,20 @@ struct ReadArgs {
     ScratchHeader *scratch;
 };
 
-constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2;
+constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarL2_128 = 3, kVarL2_256 = 4,
+              kVarBulk = 5;
+__host__ __device__ constexpr int l2_hint_of(int var) { return var == kVarL2_128 ? 128 : (var == kVarL2_256 ? 256 : 0); }
 
-template <int W, int U, bool CHECKED>
+// Per-warp state of the bulk-copy shape: a ring of U line slots and U mbarriers in shared memory
+// (32-bit shared-window addresses), and the phase parity each barrier will complete next.
+struct BulkRing {
+    uint32_t ring, bars, phases;
+    uint32_t *status;
+};
+constexpr uint32_t kBulkWaitPolls = 1u << 20;  // per line; each poll may itself sleep a little
+constexpr uint32_t kStatusBulkTimeout = 2u;    // status bit: a bulk copy did not complete in time
+
+template <int W, int U, bool CHECKED, int HINT>
 __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, uint64_t region_bytes,
                                            uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
@@ -112,7 +124,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
                 return;
             }
         }
-        load_lane<W>(lane_ptr + (uint64_t)line * (128u * W), dst);
+        load_lane<W, HINT>(lane_ptr + (uint64_t)line * (128u * W), dst);
     };
     auto fold = [&](const uint32_t(&src)[W]) {
 #pragma unroll
@@ -248,18 +260,134 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     S = s;
 }
 
+// Bulk-copy shape: lane 0 asks the copy engine for each whole line (cp.async.bulk into the warp's
+// ring in shared memory, completion counted on an mbarrier), the lanes then fold the line from
+// shared memory.  One request per line instead of 32 lane requests; same lines, same words.
+// Every wait is bounded: a copy that does not complete sets kStatusBulkTimeout, the warp stops
+// issuing, waits (bounded again) for what is still in flight and returns what it has.
+template <int W, int U>
+__device__ __forceinline__ void warp_reads_bulk(const char *__restrict__ buf, uint64_t key,
+                                                IndexSpec ix, uint64_t v, uint64_t V,
+                                                uint64_t first, uint64_t reads, uint32_t base,
+                                                uint32_t n, uint32_t lane, uint32_t &X, uint32_t &S,
+                                                BulkRing &br)
+{
+    static_assert(U >= 1 && U <= 16 && (32 % U) == 0, "ring depth must divide a batch");
+    constexpr uint32_t kLine = 128u * W;
+    LineSource src;
+    src.init(base, n, ix);
+    uint32_t x = 0, s = 0;
+    uint32_t inflight = 0;  // slots with a copy in flight (warp-uniform)
+    bool dead = false;      // a wait ran out (warp-uniform)
+
+    auto gen = [&](uint64_t i) -> uint32_t {
+        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        return src.base + mod_exact(r, src.div);
+    };
+    auto issue = [&](uint32_t line, int slot) {
+        if (lane == 0) {
+            const uint32_t bar = br.bars + 8u * slot;
+            mbar_expect_tx(bar, kLine);
+            bulk_load(br.ring + kLine * slot, buf + (uint64_t)line * kLine, kLine, bar);
+        }
+        inflight |= 1u << slot;
+    };
+    auto wait = [&](int slot) -> bool {
+        const uint32_t bar = br.bars + 8u * slot, parity = (br.phases >> slot) & 1u;
+        bool ok = false;
+        for (uint32_t k = 0; k < kBulkWaitPolls && !ok; ++k) ok = mbar_try_wait(bar, parity);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        br.phases ^= 1u << slot;  // the barrier is left to its fate if the wait ran out
+        inflight &= ~(1u << slot);
+        return ok;
+    };
+    auto consume = [&](int slot) {
+        if (!wait(slot)) {
+            dead = true;
+            if (lane == 0) atomicOr(br.status, kStatusBulkTimeout);
+            return;
+        }
+        uint32_t d[W];
+        lds_lane(br.ring + kLine * slot + lane * (4u * W), d);
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            x ^= d[w];
+            s += d[w];
+        }
+    };
+
+    const uint64_t n_batches = (reads + 31) >> 5;
+    src.enter(first, ix);
+    uint32_t cur = gen(first + lane);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u);
+        if ((uint64_t)u < reads) issue(line, u);
+    }
+    for (uint64_t b = 0; b < n_batches; ++b) {
+        const uint64_t t0 = b << 5;
+        src.enter(first + t0 + 32, ix);
+        const uint32_t nxt = gen(first + t0 + 32 + lane);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const uint64_t t = t0 + j;
+            if (t < reads && !dead) consume(j % U);
+            uint32_t line = (j + U < 32) ? __shfl_sync(0xFFFFFFFFu, cur, (j + U) & 31)
+                                         : __shfl_sync(0xFFFFFFFFu, nxt, (j + U) & 31);
+            __syncwarp();  // every lane has read the slot before the copy engine may overwrite it
+            if (t + U < reads && !dead) issue(line, j % U);
+        }
+        cur = nxt;
+        if (dead) break;
+    }
+    if (dead)  // bounded wait for the copies still in flight: shared memory must outlive them
+        for (int u = 0; u < U; ++u)
+            if (inflight & (1u << u)) wait(u);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        x ^= __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    }
+    X = x;
+    S = s;
+}
+
 template <int W, int U, int VAR>
 __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
                                            uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
-                                           uint32_t &S, uint32_t *violations)
+                                           uint32_t &S, uint32_t *violations, BulkRing &br)
 {
     if constexpr (VAR == kVarPacked && W < 4)
         warp_reads_packed<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S);
+    else if constexpr (VAR == kVarBulk)
+        warp_reads_bulk<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S, br);
     else
-        warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, ix, v, V, first,
-                                                   reads, base, n, lane, X, S, violations);
+        warp_reads_lines<W, U, VAR == kVarChecked, l2_hint_of(VAR)>(
+            buf, region_bytes, key, ix, v, V, first, reads, base, n, lane, X, S, violations);
+}
+
+// Dynamic shared memory: ballast that keeps one block per SM, and the bulk shape's rings.
+extern __shared__ __align__(128) unsigned char rr_dyn_smem[];
+
+template <int W, int U, int VAR>
+__device__ __forceinline__ BulkRing make_bulk_ring(uint32_t warp, uint32_t lane, uint32_t wpc,
+                                                   uint32_t *status)
+{
+    BulkRing br{0u, 0u, 0u, status};
+    if constexpr (VAR == kVarBulk) {
+        const uint32_t base = smem_addr(rr_dyn_smem);
+        br.ring = base + warp * (U * 128u * W);
+        br.bars = base + wpc * (U * 128u * W) + warp * (U * 8u);
+        if (lane == 0) {
+            for (int u = 0; u < U; ++u) mbar_init(br.bars + 8u * u, 1u);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncwarp();
+    }
+    return br;
 }
 
 template <int W, int U, int VAR>
@@ -271,6 +399,7 @@ __global__ void __launch_bounds__(1024, 1)
     __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     ScratchHeader *sc = a.scratch;
+    BulkRing br = make_bulk_ring<W, U, VAR>(warp, lane, a.wpc, &sc->status);
 
     if (a.mode == RR_MODE_POOLED) {
         // Work sharing inside an SM group: items (logical warp, block of reads) come from the
@@ -329,7 +458,7 @@ __global__ void __launch_bounds__(1024, 1)
                 uint32_t X, S;
                 warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix,
                                           v, a.n_warps, a.first_read + i0, n_seg, base, n, lane, X,
-                                          S, &sc->violations);
+                                          S, &sc->violations, br);
                 if (lane == 0) {
                     atomicXor(&out_words[2 * v], X);
                     atomicAdd(&out_words[2 * v + 1], S);
@@ -375,7 +504,7 @@ __global__ void __launch_bounds__(1024, 1)
         ix.sm = sm;
         ix.nsm = a.nsm;
         warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), ix, v, V, a.first_read,
-                              a.reads, base, n, lane, X, S, &sc->violations);
+                              a.reads, base, n, lane, X, S, &sc->violations, br);
         if (lane == 0) a.out[v] = make_uint2(X, S);
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -395,7 +524,7 @@ __global__ void __launch_bounds__(1024, 1)
             uint32_t X, S;
             warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
                                       a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
-                                      &sc->violations);
+                                      &sc->violations, br);
             if (lane == 0) a.out[v] = make_uint2(X, S);
         }
         __syncthreads();
@@ -444,10 +573,11 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     if (threadIdx.x == 0) t_start = globaltimer();
     const uint64_t v = (uint64_t)sm * a.wps + warp;
     uint32_t X, S;
+    BulkRing no_ring{0u, 0u, 0u, nullptr};
     warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
                                        IndexSpec{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u}, v,
                                        (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
-                                       a.n_lines, lane, X, S, nullptr);
+                                       a.n_lines, lane, X, S, nullptr, no_ring);
     if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -473,6 +603,19 @@ static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
         RR_PACKED_ROW(2)
 #undef RR_PACKED_ROW
     }
+    if (variant == RR_VARIANT_L2_128 || variant == RR_VARIANT_L2_256 ||
+        variant == RR_VARIANT_BULK) {  // comparison variants: ring depth 4 or 8 only
+#define RR_CMP_ROW(W_)                                                                  \
+    if (W == W_) {                                                                      \
+        if (variant == RR_VARIANT_L2_128) return read_kernel<W_, 8, kVarL2_128>;        \
+        if (variant == RR_VARIANT_L2_256) return read_kernel<W_, 8, kVarL2_256>;        \
+        return U == 4 ? read_kernel<W_, 4, kVarBulk> : read_kernel<W_, 8, kVarBulk>;    \
+    }
+        RR_CMP_ROW(1)
+        RR_CMP_ROW(2)
+        RR_CMP_ROW(4)
+#undef RR_CMP_ROW
+    }
     const bool checked = variant == RR_VARIANT_LDG_CHECKED;
 #define RR_ROW(W_, UMAX_)                                                               \
     if (W == W_) {                                                                      \
@@ -491,6 +634,13 @@ static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
     return nullptr;
 }
 
+// Shared memory the bulk shape needs: per warp a ring of U lines and U mbarriers.
+static size_t bulk_smem_bytes(uint32_t variant, uint32_t W, uint32_t U, uint32_t warps_per_block)
+{
+    if (variant != RR_VARIANT_BULK) return 0;
+    return (size_t)warps_per_block * U * (128u * W + 8u);
+}
+
 static bool width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
 
 struct Geometry {
@@ -505,7 +655,7 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
 {
     if (!p || !out || !scratch || !p->buf) return RR_ERR_ARG;
     if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_POOLED ||
-        p->index_mode > RR_INDEX_PHASED || p->variant > RR_VARIANT_PACKED)
+        p->index_mode > RR_INDEX_PHASED || p->variant > RR_VARIANT_BULK)
         return RR_ERR_ARG;
     if (p->reserved) return RR_ERR_ARG;
     if (p->index_mode == RR_INDEX_PHASED) {
@@ -519,6 +669,9 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_PACKED ? 4u : 8u);
     if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && p->variant == RR_VARIANT_PACKED))
         return RR_ERR_ARG;
+    if ((p->variant == RR_VARIANT_L2_128 || p->variant == RR_VARIANT_L2_256) && U != 8)
+        return RR_ERR_ARG;
+    if (p->variant == RR_VARIANT_BULK && U != 4 && U != 8) return RR_ERR_ARG;
     if (U * p->words_per_lane > 32) U = 32 / p->words_per_lane;  // the ring holds 32 words a lane
     *unroll = U;
     if ((uintptr_t)p->buf % 512u) return RR_ERR_ALIGN;
@@ -597,23 +750,64 @@ static int32_t geometry(const rr_read_params_t *p, const DeviceFacts &f, Geometr
     return RR_OK;
 }
 
+// ---- launch configuration, found once per (device, kernel, block size, blocks per SM) -----------
 // Smallest dynamic shared-memory request that makes exactly `want` blocks of `block` threads
-// resident per SM, so that a grid of nsm*want blocks puts `want` on every SM.
-template <typename K>
-static int32_t ballast_for_occupancy(K kernel, int block, int want, const DeviceFacts &f,
-                                     size_t *smem_out)
+// resident per SM (so that a grid of nsm*want blocks puts `want` on every SM), raised to `need`
+// when the kernel really uses dynamic shared memory.  The occupancy search costs ~100 runtime
+// calls, so its result is kept for the life of the process; later launches of the same
+// configuration make no occupancy or attribute call at all.
+struct LaunchKey {
+    int device;
+    const void *kernel;
+    int block, want;
+    size_t need;
+    bool operator==(const LaunchKey &o) const
+    {
+        return device == o.device && kernel == o.kernel && block == o.block && want == o.want &&
+               need == o.need;
+    }
+};
+struct LaunchEntry {
+    LaunchKey key;
+    size_t smem;
+};
+static std::mutex g_launch_mutex;
+static std::vector<LaunchEntry> g_launch_cache;
+static std::atomic<uint64_t> g_n_occupancy_queries{0}, g_n_attribute_sets{0}, g_n_event_creates{0};
+
+static int32_t search_ballast(const void *kernel, int block, int want, size_t need,
+                              const DeviceFacts &f, size_t *smem_out)
 {
     cudaFuncAttributes fa;
     RR_CUDA(cudaFuncGetAttributes(&fa, kernel));
     const int per_block_reserved = 1024;
-    int lo = f.smem_per_sm / (want + 1) - per_block_reserved - (int)fa.sharedSizeBytes + 1;
+    const int stat = (int)fa.sharedSizeBytes;
+    int lo = f.smem_per_sm / (want + 1) - per_block_reserved - stat + 1;
     if (lo < 0) lo = 0;
-    const int hi = std::min(f.smem_per_block_optin - (int)fa.sharedSizeBytes,
-                            f.smem_per_sm / want - per_block_reserved - (int)fa.sharedSizeBytes);
-    for (int smem = lo; smem <= hi; smem += 1024) {
-        RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int hi = std::min(f.smem_per_block_optin - stat,
+                            f.smem_per_sm / want - per_block_reserved - stat);
+    if ((int)need > hi) {
+        set_cuda_error(cudaErrorLaunchOutOfResources, "shared-memory ring does not fit");
+        return RR_ERR_CUDA;
+    }
+    // one opt-in to the largest request any configuration of this kernel may make; the attribute
+    // is a permission, it does not change residency
+    g_n_attribute_sets.fetch_add(1);
+    RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 std::max(hi, 0)));
+    auto blocks_at = [&](size_t smem, int *nb) -> int32_t {
+        g_n_occupancy_queries.fetch_add(1);
+        RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, kernel, block, smem));
+        return RR_OK;
+    };
+    if (want <= 0) {  // no residency requirement (LOGICAL mode): just the ring
+        *smem_out = need;
+        return RR_OK;
+    }
+    for (int smem = std::max(lo, (int)need); smem <= hi; smem += 1024) {
         int nb = 0;
-        RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, block, (size_t)smem));
+        int32_t rc = blocks_at((size_t)smem, &nb);
+        if (rc != RR_OK) return rc;
         if (nb == want) {
             *smem_out = (size_t)smem;
             return RR_OK;
@@ -622,13 +816,55 @@ static int32_t ballast_for_occupancy(K kernel, int block, int want, const Device
     }
     // registers or threads already limit residency below `want`
     int nb = 0;
-    RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, block, 0));
+    int32_t rc = blocks_at(need, &nb);
+    if (rc != RR_OK) return rc;
     if (nb == want) {
-        *smem_out = 0;
+        *smem_out = need;
         return RR_OK;
     }
     set_cuda_error(cudaErrorLaunchOutOfResources, "cannot force the requested blocks per SM");
     return RR_ERR_CUDA;
+}
+
+template <typename K>
+static int32_t launch_smem(K kernel, int block, int want, size_t need, const DeviceFacts &f,
+                           size_t *smem_out)
+{
+    const LaunchKey key{f.device, (const void *)kernel, block, want, need};
+    std::lock_guard<std::mutex> lock(g_launch_mutex);
+    for (const LaunchEntry &e : g_launch_cache)
+        if (e.key == key) {
+            *smem_out = e.smem;
+            return RR_OK;
+        }
+    size_t smem = 0;
+    int32_t rc = search_ballast((const void *)kernel, block, want, need, f, &smem);
+    if (rc != RR_OK) return rc;
+    g_launch_cache.push_back(LaunchEntry{key, smem});
+    *smem_out = smem;
+    return RR_OK;
+}
+
+// Two timing events per host thread and device, created on first use and kept.
+struct EventPair {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+};
+static int32_t timing_events(int device, EventPair **out)
+{
+    constexpr int kMaxDev = 64;
+    static thread_local EventPair pairs[kMaxDev];
+    if (device < 0 || device >= kMaxDev) return RR_ERR_UNSUPPORTED;
+    EventPair &p = pairs[device];
+    if (!p.e0) {
+        g_n_event_creates.fetch_add(1);
+        RR_CUDA(cudaEventCreate(&p.e0));
+    }
+    if (!p.e1) {
+        g_n_event_creates.fetch_add(1);
+        RR_CUDA(cudaEventCreate(&p.e1));
+    }
+    *out = &p;
+    return RR_OK;
 }
 
 // Kernel arguments of one read launch from the caller's parameters and the launch geometry.
@@ -702,6 +938,7 @@ static int32_t decode(const rr_read_params_t *p, const Geometry &g, const Device
     res->violations = h.violations;
     res->sms_covered = covered;
     res->blocks_run = h.blocks_run;
+    if (h.status & kStatusBulkTimeout) return RR_ERR_TIMEOUT;
     if (uncovered) return RR_ERR_SM_UNCOVERED;
     if (h.violations) return RR_ERR_CHECK;
     if (h.status) return RR_ERR_SM_UNCOVERED;
@@ -729,8 +966,10 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     cudaStream_t stream = (cudaStream_t)stream_;
 
     size_t smem = 0;
-    if (p->mode != RR_MODE_LOGICAL) {
-        rc = ballast_for_occupancy(kernel, (int)g.block, (int)g.cps, f, &smem);
+    const size_t need = bulk_smem_bytes(p->variant, p->words_per_lane, U, g.wpc);
+    if (p->mode != RR_MODE_LOGICAL || need) {
+        rc = launch_smem(kernel, (int)g.block, p->mode != RR_MODE_LOGICAL ? (int)g.cps : 0, need, f,
+                         &smem);
         if (rc != RR_OK) return rc;
     }
 
@@ -738,49 +977,31 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     Tables tab;
     make_launch_args(p, g, f, out_dev, scratch_dev, &a, &tab);
 
-    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    EventPair *ev = nullptr;
     if (res) {
-        RR_CUDA(cudaEventCreate(&e0));
-        RR_CUDA(cudaEventCreate(&e1));
+        rc = timing_events(f.device, &ev);
+        if (rc != RR_OK) return rc;
     }
-    auto cleanup = [&]() {
-        if (e0) cudaEventDestroy(e0);
-        if (e1) cudaEventDestroy(e1);
-        e0 = e1 = nullptr;
-    };
-#define RR_CUDA_C(call)                        \
-    do {                                       \
-        cudaError_t e__ = (call);              \
-        if (e__ != cudaSuccess) {              \
-            set_cuda_error(e__, #call);        \
-            cleanup();                         \
-            return RR_ERR_CUDA;                \
-        }                                      \
-    } while (0)
-
     // claims, status, records -- and, in pooled mode, the work counters behind them
-    RR_CUDA_C(cudaMemsetAsync(scratch_dev, 0,
-                              p->mode == RR_MODE_POOLED ? sizeof(ScratchHeader)
-                                                        : offsetof(ScratchHeader, probe),
-                              stream));
+    RR_CUDA(cudaMemsetAsync(scratch_dev, 0,
+                            p->mode == RR_MODE_POOLED ? sizeof(ScratchHeader)
+                                                      : offsetof(ScratchHeader, probe),
+                            stream));
     if (p->mode == RR_MODE_PER_SM && g.active_sms != (uint32_t)f.nsm)
-        RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
+        RR_CUDA(cudaMemsetAsync(out_dev, 0, (size_t)f.nsm * g.wps * sizeof(uint2), stream));
     if (p->mode == RR_MODE_POOLED)  // the checksums the atomics add into
-        RR_CUDA_C(cudaMemsetAsync(out_dev, 0, (size_t)p->n_warps * sizeof(uint2), stream));
-    if (res) RR_CUDA_C(cudaEventRecord(e0, stream));
+        RR_CUDA(cudaMemsetAsync(out_dev, 0, (size_t)p->n_warps * sizeof(uint2), stream));
+    if (res) RR_CUDA(cudaEventRecord(ev->e0, stream));
     kernel<<<g.grid, g.block, smem, stream>>>(a, tab);
-    RR_CUDA_C(cudaGetLastError());
+    RR_CUDA(cudaGetLastError());
     if (!res) return RR_OK;
-    RR_CUDA_C(cudaEventRecord(e1, stream));
-    RR_CUDA_C(cudaEventSynchronize(e1));
-    float ms = 0.f;
-    RR_CUDA_C(cudaEventElapsedTime(&ms, e0, e1));
+    RR_CUDA(cudaEventRecord(ev->e1, stream));
     static thread_local ScratchHeader h;
-    RR_CUDA_C(cudaMemcpyAsync(&h, scratch_dev, offsetof(ScratchHeader, probe),
-                              cudaMemcpyDeviceToHost, stream));
-    RR_CUDA_C(cudaStreamSynchronize(stream));
-    cleanup();
-#undef RR_CUDA_C
+    RR_CUDA(cudaMemcpyAsync(&h, scratch_dev, offsetof(ScratchHeader, probe),
+                            cudaMemcpyDeviceToHost, stream));
+    RR_CUDA(cudaStreamSynchronize(stream));
+    float ms = 0.f;
+    RR_CUDA(cudaEventElapsedTime(&ms, ev->e0, ev->e1));
     return decode(p, g, f, h, (double)ms * 1e-3, res);
 }
 
@@ -819,6 +1040,16 @@ extern "C" int32_t rr_read_block_times(const void *scratch_dev, uint32_t nsm, ui
         t_start[s] = h.rec[s].t_end ? h.rec[s].t_start : 0;
         t_end[s] = h.rec[s].t_end;
     }
+    return RR_OK;
+}
+
+extern "C" int32_t rr_host_counters(rr_host_counters_t *out)
+{
+    if (!out) return RR_ERR_ARG;
+    out->occupancy_queries = g_n_occupancy_queries.load();
+    out->attribute_sets = g_n_attribute_sets.load();
+    out->event_creates = g_n_event_creates.load();
+    out->device_fact_queries = device_fact_queries();
     return RR_OK;
 }
 
@@ -893,14 +1124,15 @@ extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_
     if (sm_a >= (uint32_t)f.nsm || sm_b >= (uint32_t)f.nsm) return RR_ERR_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    rc = ballast_for_occupancy(probe_kernel, (int)wps * 32, 1, f, &smem);
+    rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
     if (rc != RR_OK) return rc;
     ProbeRecord *rec = &((ScratchHeader *)scratch_dev)->probe;
     ProbeArgs pa = probe_args(buf, region_bytes, sm_a, sm_b, total_reads, wps, seed, out_dev, rec,
                               f.nsm);
-    cudaEvent_t e0, e1;
-    RR_CUDA(cudaEventCreate(&e0));
-    RR_CUDA(cudaEventCreate(&e1));
+    EventPair *ev = nullptr;
+    rc = timing_events(f.device, &ev);
+    if (rc != RR_OK) return rc;
+    cudaEvent_t e0 = ev->e0, e1 = ev->e1;
     int32_t result = RR_ERR_SM_UNCOVERED;
     std::memset(res, 0, sizeof(*res));
     for (int attempt = 0; attempt < 3 && result == RR_ERR_SM_UNCOVERED; ++attempt) {
@@ -934,8 +1166,6 @@ extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_
             result = RR_OK;
         }
     }
-    cudaEventDestroy(e0);
-    cudaEventDestroy(e1);
     return result;
 }
 
@@ -958,7 +1188,7 @@ extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint6
     if (nsm != (uint32_t)f.nsm) return RR_ERR_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    rc = ballast_for_occupancy(probe_kernel, (int)wps * 32, 1, f, &smem);
+    rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
     if (rc != RR_OK) return rc;
 
     const size_t n_pairs = (size_t)nsm * (nsm + 1) / 2;
@@ -1079,8 +1309,9 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     if (rc != RR_OK) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    if (p->mode == RR_MODE_PER_SM) {
-        rc = ballast_for_occupancy(kernel, (int)g.block, 1, f, &smem);
+    const size_t need = bulk_smem_bytes(p->variant, p->words_per_lane, U, g.wpc);
+    if (p->mode == RR_MODE_PER_SM || need) {
+        rc = launch_smem(kernel, (int)g.block, p->mode == RR_MODE_PER_SM ? 1 : 0, need, f, &smem);
         if (rc != RR_OK) return rc;
     }
     ReadArgs a;

@@ -167,6 +167,47 @@ class Session:
         rates = sorted(r.gbps for r in res)
         return rates[(len(rates) - 1) // 2], res[-1]
 
+    def sustained(self, p: rr.ReadParams, out=None, *, settle: int = 150, min_ms: float = 50.0,
+                  reps: int = 5, sampler=None) -> dict:
+        """The one measurement protocol every arm of a comparison goes through: `settle` untimed
+        launches of the very same call (clocks and caches reach their sustained state), then
+        `reps` timed regions, each a run of back-to-back asynchronous launches long enough to
+        hold at least `min_ms` of kernel time, bracketed by CUDA events on the launching stream.
+        Returns median / min / max GB/s over the regions, the launches per region and, with a
+        clocks.ClockSampler, the SM clock and power seen while the regions ran."""
+        import time
+        t = self.torch
+        out = self.out if out is None else out
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+
+        def region(n):
+            e0.record()
+            for _ in range(n):
+                rr.rr_random_read(p, out, self.scratch, timed=False)
+            e1.record()
+            t.cuda.synchronize()
+            return e0.elapsed_time(e1)
+
+        region(max(1, settle))
+        probe_n = 4
+        per_launch_ms = max(region(probe_n) / probe_n, 1e-3)
+        n = max(1, int(np.ceil(min_ms / per_launch_ms)))
+        rep = rr.rr_read_report(p, self.scratch)          # also checks coverage and status
+        t_begin = time.time()
+        ms = [region(n) for _ in range(max(1, reps))]
+        t_end = time.time()
+        rates = sorted(rep.bytes * n / m * 1e-6 for m in ms)
+        res = {"gbps": rates[(len(rates) - 1) // 2], "gbps_min": rates[0], "gbps_max": rates[-1],
+               "launches_per_region": n, "regions": len(ms), "ms_per_region": float(np.median(ms)),
+               "bytes_per_launch": int(rep.bytes), "settle_launches": settle}
+        if sampler is not None:
+            c = sampler.window(t_begin, t_end)
+            res["sm_mhz"], res["power_w"], res["clock_reasons"] = (c["sm_mhz"], c["power_w"],
+                                                                   c["reasons"])
+            if c["sm_mhz"]:
+                res["gbps_per_sm_ghz"] = res["gbps"] / (c["sm_mhz"] * 1e-3)
+        return res
+
     def checksums(self, n: int) -> np.ndarray:
         return self.out[:n].cpu().numpy().view(np.uint32)
 

@@ -61,6 +61,23 @@ def test_pooled_equals_per_warp_definition():
             assert base <= oracle.line(23, v, i, base, n) < base + n      # inside the window
 
 
+def test_pooled_with_148_groups_and_empty_groups_equals_per_warp_definition():
+    """One window per SM (148 groups of ~32 warps) and groups that own no warps: the single loop
+    over all warps must find each warp's owner, skipping empty ranges."""
+    region = 148 * 5000 * 128
+    win, ws = oracle.make_weighted_windows(region, 1, [900 + 7 * (g % 11) for g in range(148)], 4736)
+    out = oracle.read_pooled(region, 1, win, ws, reads=5, seed=23, first_read=2)
+    for v in list(range(0, 4736, 97)) + [4735]:
+        g = int(np.searchsorted(ws, v, side="right") - 1)
+        assert tuple(out[v]) == oracle.warp_checksum(23, v, 2, 5, 1, int(win[g, 0]), int(win[g, 1]))
+    win = np.array([[0, 100], [100, 50], [150, 70], [300, 10]], np.uint32)
+    ws = [0, 0, 6, 6, 9]                                   # groups 0 and 2 own nothing
+    out = oracle.read_pooled(1 << 20, 1, win, ws, reads=7, seed=3)
+    for v in range(9):
+        g = 1 if v < 6 else 3
+        assert tuple(out[v]) == oracle.warp_checksum(3, v, 0, 7, 1, int(win[g, 0]), int(win[g, 1]))
+
+
 def test_pooled_with_one_group_is_the_logical_mode():
     region = 3 << 20
     L = region // 128
