@@ -25,6 +25,8 @@
  *   r(seed,v,i)  = sm64(k_v + i * 0x9E3779B97F4A7C15)      -- i-th draw of warp v
  *   line(v,i)    = base + (r mod n)   for a window of n lines starting at line `base`
  *                  (RR_INDEX_STRIDE: base + ((i * V + v) mod n), V = warps in the call)
+ *                  (RR_INDEX_MIXED, period k: read i with i mod k == 0 is read i/k of the warp's
+ *                  sequential walk, base + (((i/k) * V + v) mod n); other reads are random)
  *                  (RR_INDEX_PHASED: the window is cut into Q = ceil(n / sub) sub-windows
  *                  [floor(n q / Q), floor(n (q+1) / Q)), sub = phase_window_bytes / (128 W);
  *                  read i belongs to phase p = floor(i / phase_reads) and draws
@@ -69,6 +71,7 @@ extern "C" {
 #define RR_INDEX_RANDOM 0u
 #define RR_INDEX_STRIDE 1u
 #define RR_INDEX_PHASED 2u /* random inside a sub-window that moves with the read counter         */
+#define RR_INDEX_MIXED 3u  /* every mix_period-th read sequential, the others random              */
 #define RR_VARIANT_LDG 0u         /* ld.global.nc.L1::no_allocate vector loads                  */
 #define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
 #define RR_VARIANT_PACKED 2u      /* every lane loads 16 bytes: one warp load covers 4/W lines  */
@@ -77,6 +80,8 @@ extern "C" {
 #define RR_VARIANT_L2_256 4u      /* RR_VARIANT_LDG with the .L2::256B prefetch qualifier       */
 #define RR_VARIANT_BULK 5u        /* one cp.async.bulk per line into a ring in shared memory,   */
                                   /* completion on an mbarrier, lanes fold from shared memory   */
+#define RR_VARIANT_SORTED 6u      /* RR_VARIANT_PACKED with each warp's reads taken in an order */
+                                  /* that keeps the SM inside one part of its window at a time  */
 
 const char *rr_strerror(int32_t code);
 const char *rr_last_cuda_error(void);
@@ -99,7 +104,10 @@ int32_t rr_host_counters(rr_host_counters_t *out /*HOST*/);
 
 /* ---- device facts ------------------------------------------------------------------------
  * Paper, Section 1.1: the %smid / %nsmid registers are the only layout facts a program gets.
- * Fills *out (HOST) for the current device.  nsm_reg is %nsmid read by a one-thread kernel.
+ * Fills *out (HOST) for the current device.  nsm_reg is %nsmid, read by a one-thread kernel that
+ * runs on `stream` and writes its answer into the first word of scratch_dev (DEVICE, 16-byte
+ * aligned, at least 4 bytes; rr_scratch_bytes() will do); with scratch_dev == NULL nothing is
+ * launched and nsm_reg stays 0.  Synchronises `stream` when it launches.
  * theoretical_gbps = 2 * memory clock * bus width / 8.                                        */
 typedef struct {
     uint32_t nsm_prop;       /* cudaDeviceProp::multiProcessorCount                            */
@@ -113,7 +121,8 @@ typedef struct {
     char name[64];
     char uuid[40];           /* 32 hex digits, NUL-terminated                                  */
 } rr_device_info_t;
-int32_t rr_device_info(rr_device_info_t *out /*HOST*/);
+int32_t rr_device_info(rr_device_info_t *out /*HOST*/, void *scratch_dev /*DEVICE or NULL*/,
+                       void *stream);
 
 /* ---- scratch ------------------------------------------------------------------------------
  * Bytes of DEVICE scratch rr_random_read / rr_probe_pair / rr_cluster need (claim table,
@@ -128,9 +137,10 @@ size_t rr_scratch_bytes(void);
 int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
 
 /* ---- random line reads -------------------------------------------------------------------
- * Paper, Section 2.1 ("every warp reads random coalesced arrays of 32 32-bit words in a memory
- * region of varying size"; 64- and 128-bit words), Section 2.1 second experiment and Section
- * 2.4 (all warps of an SM / of an SM group read inside one chunk).
+ * Paper, Section 2.1, Fig. 1 (the basic benchmark: each warp fetches whole lines of 32 words at
+ * random positions of a region whose size is varied; 32-, 64- and 128-bit words), Section 2.1
+ * second experiment and Section 2.4, Fig. 6 (all warps of an SM / of an SM group read inside
+ * one chunk).
  *
  * The region is the prefix [0, region_bytes) of buf; L = floor(region_bytes / (128*W)) lines.
  * RR_MODE_LOGICAL: n_warps logical warps, each reading the whole region; any block may run
@@ -158,6 +168,16 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   sub-window at a time while a whole cycle of phases still covers the window uniformly.
  *   SMs that share a window (the whole region when group_of_sm is NULL) start their cycles at
  *   staggered sub-windows, so the region can also be read from every SM with no partition.
+ * RR_INDEX_MIXED (LOGICAL and PER_SM modes; Section 2.1 closes on sequential access being the
+ *   faster kind): a blend of the two, one read in mix_period sequential, to place a workload
+ *   between the random rate and the sequential ceiling.  mix_period = 1 is RR_INDEX_STRIDE.
+ * RR_VARIANT_SORTED (W = 1, 2; RR_INDEX_RANDOM): the checksums do not depend on the order of a
+ *   warp's reads, so the kernel is free to choose one.  This variant cuts the stream into epochs
+ *   of sort_parts * sort_reads reads and performs the reads of an epoch part by part of the
+ *   warp's window (sort_parts equal parts): at any moment an SM then works inside 1/sort_parts of
+ *   its window, which its own translation cache can hold, although the window -- the set of lines
+ *   the warp may read, Section 1.3 -- is unchanged and static.  Results are those of
+ *   RR_VARIANT_PACKED bit for bit; the price is sort_parts hashes per read.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
@@ -192,8 +212,11 @@ typedef struct {
     uint32_t pool_block_reads;  /* POOLED: smallest grab in reads, 0 = 64; else must be 0      */
     const uint32_t *warp_start; /* POOLED: HOST [n_groups+1]; else NULL                        */
     uint32_t phase_reads;       /* RR_INDEX_PHASED: reads per phase, a power of two >= 32      */
-    uint32_t reserved;          /* must be 0                                                   */
+    uint32_t mix_period;        /* RR_INDEX_MIXED: a power of two in [1, 2^20]; else must be 0  */
     uint64_t phase_window_bytes; /* RR_INDEX_PHASED: largest sub-window                        */
+    uint32_t sort_parts;        /* RR_VARIANT_SORTED: parts of the window, a power of two 2..64 */
+    uint32_t sort_reads;        /* RR_VARIANT_SORTED: reads per part and epoch, a multiple of  */
+                                /* 32 (1024 is a good value); both 0 for every other variant   */
 } rr_read_params_t;
 
 typedef struct {
@@ -253,8 +276,8 @@ int32_t rr_random_read_static(const rr_read_params_t *params /*HOST*/, void *out
                               rr_result_t *res /*HOST or NULL*/, void *stream);
 
 /* ---- two-SM contention probe ---------------------------------------------------------------
- * Paper, Section 2.2: "if we run our memory access kernel with only two SMs, we expect ... a
- * drop in throughput when those SMs are in the same GPC".  A full grid is launched; blocks exit
+ * Paper, Section 2.2, Fig. 2: the read kernel is run on two SMs only; a pair that shares a
+ * translation resource is expected to lose throughput.  A full grid is launched; blocks exit
  * unless they are the first block on sm_a or sm_b.  Each surviving SM performs total_reads/2
  * random 128-byte line reads (W = 1) over the whole region with warps_per_sm warps (1..32;
  * total_reads must be a multiple of 2*warps_per_sm), warp ids and streams as in RR_MODE_PER_SM.
@@ -274,15 +297,51 @@ size_t rr_probe_matrix_scratch_bytes(uint32_t nsm);
 /* All unordered pairs and all solos: T_host[a*nsm+b] = T_host[b*nsm+a] = pair GB/s (median of
  * `repeats` sweeps, repeats >= 1), T_host[a*nsm+a] = solo GB/s.  Launches are queued back to
  * back per sweep and read back once.  out_dev as in rr_probe_pair (overwritten by every pair).
- * overlap_min_host (HOST, may be NULL) receives the smallest overlap fraction
- * (earliest end - latest start) / (latest end - earliest start) over all pairs.              */
+ *
+ * The two SMs of a pair must read side by side for the figure to mean contention, so (i) the
+ * first of the two blocks to arrive waits (at most 0.2 ms) for the other before it starts, and
+ * (ii) a pair whose overlap fraction
+ *   (earliest end - latest start) / (latest end - earliest start)
+ * is below 0.98 is measured again on its own with twice the reads, up to three doublings and
+ * only while a doubling still raises the overlap by 0.01 (two SMs of different speed never
+ * reach 0.98 however long they run); the sample with the best overlap is kept.
+ * stats (HOST, may be NULL): the smallest kept overlap, how many pairs stayed below 0.98 in
+ * some sweep, how many extra launches the rule cost.  overlap_host (HOST nsm*nsm float, may be
+ * NULL): per pair, the smallest kept overlap over the sweeps (diagonal 1).                    */
+typedef struct {
+    double overlap_min;        /* smallest kept overlap over all pairs and sweeps              */
+    uint32_t pairs_below_goal; /* pairs whose kept overlap stayed below 0.98 in some sweep     */
+    uint32_t reruns;           /* extra launches with more reads                               */
+    uint32_t relaunched;       /* pairs redone because an SM got no block in the queued launch */
+} rr_probe_stats_t;
 int32_t rr_probe_matrix(const void *buf /*DEVICE*/, uint64_t region_bytes, uint64_t total_reads,
                         uint32_t warps_per_sm, uint64_t seed, uint32_t repeats,
                         float *T_host /*HOST nsm*nsm*/, uint32_t nsm, void *out_dev /*DEVICE*/,
-                        void *scratch_dev /*DEVICE*/, double *overlap_min_host, void *stream);
+                        void *scratch_dev /*DEVICE*/, rr_probe_stats_t *stats /*HOST*/,
+                        float *overlap_host /*HOST*/, void *stream);
+
+/* The same for rows [row_begin, row_end) of the matrix only: pairs (a, b) with a in the range and
+ * b >= a; the entries (a, b), (b, a) and (a, a) of T_host (and overlap_host) are written, the rest
+ * left alone; stats cover these rows.  A caller can so probe a card in blocks of rows and keep
+ * what is done (the full sweep takes ~10^4 launches).  rr_probe_matrix is rows [0, nsm).       */
+int32_t rr_probe_rows(const void *buf /*DEVICE*/, uint64_t region_bytes, uint64_t total_reads,
+                      uint32_t warps_per_sm, uint64_t seed, uint32_t repeats, uint32_t row_begin,
+                      uint32_t row_end, float *T_host /*HOST nsm*nsm*/, uint32_t nsm,
+                      void *out_dev /*DEVICE*/, void *scratch_dev /*DEVICE*/,
+                      rr_probe_stats_t *stats /*HOST*/, float *overlap_host /*HOST*/, void *stream);
+
+/* The rule that turns one probe's timers into a rate (host only).  t_start, t_end (ns) and claim
+ * hold one entry per SM (two for a pair, the first only when solo = 1); an SM with claim 0 or
+ * no end time never ran: RR_ERR_SM_UNCOVERED.  gbps = bytes of the SMs that ran (total_reads/2
+ * lines of 128 bytes each) / (latest end - earliest start); overlap as defined above (1 for a
+ * solo run).                                                                                  */
+int32_t rr_probe_rate(const uint64_t *t_start, const uint64_t *t_end, const uint32_t *claim,
+                      uint32_t solo, uint64_t total_reads, double *gbps, double *seconds,
+                      double *overlap);
 
 /* ---- contention matrix -> SM groups --------------------------------------------------------
- * Paper, Section 2.2 and Figure 3 ("rearranging the indices" so groups show as blocks).  Here:
+ * Paper, Section 2.2 and Figure 3 (the SM indices are reordered until the groups show up as
+ * blocks of the matrix).  Here:
  * symmetrise, quantise against the median, average-linkage agglomeration with exact integer
  * sums, cut at the largest height gap among cuts leaving 2..n/3 clusters, null rule (gap below
  * 4 robust standard deviations of the height, or below 1 % of the median pair rate -- the paper
@@ -300,7 +359,7 @@ int32_t rr_cluster(const float *T_host, uint32_t n, uint32_t flags, void *scratc
                    double *heights_host, void *stream);
 
 /* ---- cross-check of the layout by cluster placement -----------------------------------------
- * Paper, Section 1.1: "there is no simple way to determine which GPC each SM is on".  Blocks of
+ * Paper, Section 1.1: a program is not told which GPC an SM belongs to.  Blocks of
  * one thread-block cluster always run on one GPC, so this call launches clusters of 2..8 small
  * blocks, records %smid per block and merges SMs that shared a cluster: gpc_of_sm_host[nsm]
  * (HOST) receives a GPC label per SM (numbered by smallest SM id), *n_gpcs their count.  No
@@ -312,11 +371,15 @@ int32_t rr_gpc_map(void *scratch_dev /*DEVICE*/, int32_t *gpc_of_sm_host /*HOST*
                    uint32_t *n_gpcs, uint32_t nsm, void *stream);
 
 /* ---- windows per group (host only) -------------------------------------------------------
- * Paper, Section 1.3 ("restricted to a 64GB window (or, say, half the memory for simplicity)")
- * and Section 2.4.  The L lines of the region are cut into K = ceil(L / floor(window_bytes /
- * (128*W))) chunks of floor(L/K) lines, the last running to L.  policy 0: group g takes chunk
- * g mod K.  policy 1 (the paper's naive per-SM control; pass one group per SM): chunk
- * sm64(seed ^ g) mod K.  *coverage (may be NULL) = distinct chunks used / K.                  */
+ * Paper, Section 1.3 (each group confined to a window below the reach; half of memory as the
+ * simple case) and Section 2.4.  The L lines of the region are cut into K = ceil(L /
+ * floor(window_bytes / (128*W))) chunks of floor(L/K) lines, the last running to L.
+ * policy 0: group g takes chunk g mod K.  policy 1 (the paper's naive per-SM control; pass one
+ * group per SM): chunk sm64(seed ^ g) mod K.  *coverage (may be NULL) = distinct chunks used / K.
+ * policy 2 (Section 1.3 does not ask for disjoint windows): n_groups windows of exactly
+ * S = floor(window_bytes / (128*W)) lines (clipped to [1, L]), evenly spaced and overlapping:
+ * base_g = floor(g * (L - S) / (n_groups - 1)) (0 for a single group), so the first window
+ * starts at line 0 and the last ends at line L; *coverage = lines inside some window / L.     */
 int32_t rr_make_windows(uint64_t region_bytes, uint32_t words_per_lane, uint64_t window_bytes,
                         uint32_t n_groups, uint32_t policy, uint64_t seed,
                         rr_window_t *out_host /*HOST n_groups*/, double *coverage);
@@ -337,12 +400,75 @@ int32_t rr_make_weighted_windows(uint64_t region_bytes, uint32_t words_per_lane,
                                  uint32_t *warp_start_host);
 
 /* ---- plateau, cliff and reach from a size sweep (host only) --------------------------------
- * Paper, Section 2.1 / Figure 1 ("something dramatic happens when the memory region is larger
- * than about 64GB").  size_bytes strictly increasing.  plateau = lower median of GB/s over
+ * Paper, Section 2.1 / Figure 1 (throughput collapses once the region outgrows the translation
+ * reach).  size_bytes strictly increasing.  plateau = lower median of GB/s over
  * 4 GiB <= size <= 32 GiB; a cliff exists iff a larger size has GB/s < 0.8 plateau; reach =
  * largest size before it with GB/s >= 0.9 plateau.  Returns 1 (cliff), 0 (none) or an error.  */
 int32_t rr_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
                  double *plateau, uint64_t *reach_bytes);
+
+/* Next size to measure when refining the reach (host only).  Paper, Section 2.1 / Figure 1: a
+ * sweep brackets the cliff between two of its sizes.  With good = the reach rr_reach finds in
+ * the sweep so far and bad = the smallest measured size above it, the next point is
+ * mid = floor((good + bad) / 2 / step_bytes) * step_bytes.  Returns 1 and *next_size = mid while
+ * bad - good > step_bytes and good < mid < bad; 0 (and *next_size = 0) when the refinement is
+ * finished or there is no cliff; an error code as rr_reach.  The caller measures that size,
+ * inserts the point and asks again: a point is judged by rr_reach alone.                      */
+int32_t rr_reach_next(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
+                      uint64_t step_bytes, uint64_t *next_size);
+
+/* How far one SM's own translation cache reaches (host only).  The experiment of Section 2.1
+ * with one window per SM gives a rate per window size (sizes strictly increasing).  The level
+ * small windows sustain is the middle one of the first three rates (the first rate if fewer);
+ * *reach_bytes = the last size of the leading run of points with rate >= keep * level
+ * (0 < keep <= 1); the first size if even that one falls short.                               */
+int32_t rr_sm_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points, double keep,
+                    uint64_t *reach_bytes);
+
+/* One window per SM, the SMs of a resource group side by side (host only).  Paper, Section 2.4
+ * gives each group one chunk; this finer plan gives every active SM a window id of its own,
+ * handed out group by group (groups in increasing number, SMs in increasing id), so that
+ * windows laid out in id order put the windows of a group's SMs next to each other and each
+ * group still stays inside one stretch below its reach.  group_of_sm, owner_of_sm: HOST [nsm];
+ * inactive SMs stay RR_SM_INACTIVE.  *n_owners = number of ids (= active SMs).                 */
+int32_t rr_owner_map(const uint16_t *group_of_sm, uint32_t nsm, uint16_t *owner_of_sm,
+                     uint32_t *n_owners);
+
+/* Size of the moving sub-windows of RR_INDEX_PHASED (host only): the slice an SM works through
+ * is cut into the smallest power-of-two number of parts (at most max_parts) that makes a part
+ * no larger than a quarter of the SM's reach (two phases can be live at once and should both
+ * fit with room to spare); *sub_bytes = ceil(slice_bytes / *parts).                            */
+int32_t rr_phase_window(uint64_t slice_bytes, uint64_t sm_reach_bytes, uint32_t max_parts,
+                        uint32_t *parts, uint64_t *sub_bytes);
+
+/* New capacity weights from one observed pooled run (host only).  Paper, Section 2.3: a group's
+ * throughput belongs to the group.  Group g did work[g] units and its last SM finished
+ * finish_ns[g] after the common start (0 = not seen).  In integers:
+ *   rate_g = max(1, floor(work_g * 2^48 / finish_g));  unseen groups get
+ *   max(1, smallest seen rate / 1024);  weight_g = max(1, floor((rate_g * scale + T/2) / T)),
+ *   T = sum of rates.
+ * RR_ERR_RANGE if no group finished any work.  Feed the weights to rr_make_weighted_windows,
+ * run again, repeat until rr_finish_spread_ppm is small.                                       */
+int32_t rr_rebalance_weights(const uint32_t *work, const uint64_t *finish_ns, uint32_t n_groups,
+                             uint32_t scale, uint32_t *weight);
+
+/* When each group finished, from the per-SM timers rr_read_block_times returns (host only):
+ * the common start is the earliest start over the SMs that ran; finish_ns[g] = latest end over
+ * group g's SMs that ran minus that start (at least 1; 0 if none ran); *span_ns = latest end
+ * overall minus the common start.  RR_ERR_MAP if an SM that ran names a group >= n_groups.     */
+int32_t rr_group_finish(const uint64_t *t_start, const uint64_t *t_end, const uint16_t *group_of_sm,
+                        uint32_t nsm, uint32_t n_groups, uint64_t *finish_ns, uint64_t *span_ns);
+
+/* (latest - earliest) / latest finish over the groups that ran, in parts per million, rounded
+ * down (host only).                                                                            */
+int32_t rr_finish_spread_ppm(const uint64_t *finish_ns, uint32_t n_groups, uint32_t *ppm);
+
+/* How evenly a set of windows covers the region (host only): *covered = lines inside at least
+ * one window; *depth_min / *depth_max = smallest / largest number of windows over a covered
+ * line.  With equal work and equal sizes the read density at a line is proportional to its
+ * depth, so depth_max / depth_min says how uniform overlapping windows (policy 2) are.         */
+int32_t rr_window_cover(const rr_window_t *windows, uint32_t n_groups, uint64_t n_lines,
+                        uint64_t *covered, uint32_t *depth_min, uint32_t *depth_max);
 
 #ifdef __cplusplus
 }

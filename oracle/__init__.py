@@ -68,6 +68,12 @@ def _load():
         lib.orc_read_per_sm_phased.restype = i32
         lib.orc_read_per_sm_phased.argtypes = [u64, u32, u32, u32, u64, u64, u64, p, p, p, u32, u64,
                                                u64, p]
+        lib.orc_line_mixed.restype = u64
+        lib.orc_line_mixed.argtypes = [u64, u64, u64, u64, u64, u64, u64]
+        lib.orc_warp_checksum_mixed.restype = None
+        lib.orc_warp_checksum_mixed.argtypes = [u64, u64, u64, u64, u64, u32, u64, u64, u64, p, p]
+        lib.orc_read_per_sm_mixed.restype = i32
+        lib.orc_read_per_sm_mixed.argtypes = [u64, u32, u32, u32, u64, u64, u64, p, p, p, u32, u64, p]
         lib.orc_read_logical.restype = i32
         lib.orc_read_logical.argtypes = [u64, u32, u32, u64, u64, u64, u64, p]
         lib.orc_read_logical_materialised.restype = i32
@@ -84,6 +90,24 @@ def _load():
         lib.orc_cluster.argtypes = [p, u32, u32, p, p, p, p]
         lib.orc_reach.restype = i32
         lib.orc_reach.argtypes = [p, p, u32, p, p]
+        lib.orc_reach_next.restype = i32
+        lib.orc_reach_next.argtypes = [p, p, u32, u64, p]
+        lib.orc_sm_reach.restype = i32
+        lib.orc_sm_reach.argtypes = [p, p, u32, ctypes.c_double, p]
+        lib.orc_owner_map.restype = i32
+        lib.orc_owner_map.argtypes = [p, u32, p, p]
+        lib.orc_phase_window.restype = i32
+        lib.orc_phase_window.argtypes = [u64, u64, u32, p, p]
+        lib.orc_rebalance_weights.restype = i32
+        lib.orc_rebalance_weights.argtypes = [p, p, u32, u32, p]
+        lib.orc_finish_spread_ppm.restype = i32
+        lib.orc_finish_spread_ppm.argtypes = [p, u32, p]
+        lib.orc_group_finish.restype = i32
+        lib.orc_group_finish.argtypes = [p, p, p, u32, u32, p, p]
+        lib.orc_window_cover.restype = i32
+        lib.orc_window_cover.argtypes = [p, p, u32, u64, p, p, p]
+        lib.orc_probe_rate.restype = i32
+        lib.orc_probe_rate.argtypes = [p, p, p, u32, u64, p, p, p]
         _lib = lib
     return _lib
 
@@ -222,6 +246,40 @@ def read_per_sm_phased(region_bytes: int, W: int, nsm: int, wps: int, reads: int
     return out
 
 
+def line_mixed(seed: int, v: int, i: int, base: int, n: int, mix_period: int,
+               n_warps_total: int = 1) -> int:
+    return int(_load().orc_line_mixed(seed, v, n_warps_total, i, base, n, mix_period))
+
+
+def warp_checksum_mixed(seed: int, v: int, first_read: int, reads: int, W: int, base: int, n: int,
+                        mix_period: int, n_warps_total: int = 1):
+    x = ctypes.c_uint32()
+    s = ctypes.c_uint32()
+    _load().orc_warp_checksum_mixed(seed, v, n_warps_total, first_read, reads, W, base, n,
+                                    mix_period, ctypes.byref(x), ctypes.byref(s))
+    return int(x.value), int(s.value)
+
+
+def read_per_sm_mixed(region_bytes: int, W: int, nsm: int, wps: int, reads: int, seed: int,
+                      mix_period: int, group_of_sm=None, windows=None,
+                      first_read: int = 0) -> np.ndarray:
+    """Per-SM mode where every mix_period-th read of a warp's stream is sequential."""
+    out = np.zeros((nsm * wps, 2), dtype=np.uint32)
+    g = wb = wn = None
+    ng = 0
+    if group_of_sm is not None:
+        g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+        w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+        wb = np.ascontiguousarray(w[:, 0])
+        wn = np.ascontiguousarray(w[:, 1])
+        ng = w.shape[0]
+    rc = _load().orc_read_per_sm_mixed(region_bytes, W, nsm, wps, first_read, reads, seed, _ptr(g),
+                                       _ptr(wb), _ptr(wn), ng, mix_period, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
 def make_windows(region_bytes: int, W: int, window_bytes: int, n_groups: int, policy: int = 0,
                  seed: int = 0):
     """Windows per group as (n_groups, 2) uint32 {base_line, n_lines}, and the coverage fraction."""
@@ -298,6 +356,114 @@ def reach(size_bytes, gbps):
     if rc < 0:
         raise OracleError(rc)
     return bool(rc), float(plateau.value), int(r.value)
+
+
+def reach_next(size_bytes, gbps, step_bytes: int) -> int:
+    """Next size to measure while refining the reach, or 0 when done."""
+    s = np.ascontiguousarray(size_bytes, dtype=np.uint64)
+    g = np.ascontiguousarray(gbps, dtype=np.float64)
+    nxt = ctypes.c_uint64()
+    rc = _load().orc_reach_next(_ptr(s), _ptr(g), len(s), step_bytes, ctypes.byref(nxt))
+    if rc < 0:
+        raise OracleError(rc)
+    return int(nxt.value) if rc else 0
+
+
+def sm_reach(size_bytes, gbps, keep: float = 0.97) -> int:
+    s = np.ascontiguousarray(size_bytes, dtype=np.uint64)
+    g = np.ascontiguousarray(gbps, dtype=np.float64)
+    r = ctypes.c_uint64()
+    rc = _load().orc_sm_reach(_ptr(s), _ptr(g), len(s), keep, ctypes.byref(r))
+    if rc != 0:
+        raise OracleError(rc)
+    return int(r.value)
+
+
+def owner_map(group_of_sm):
+    """(owner_of_sm uint16[nsm], n_owners): one window id per active SM, group by group."""
+    g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+    out = np.zeros(g.shape[0], dtype=np.uint16)
+    n = ctypes.c_uint32()
+    rc = _load().orc_owner_map(_ptr(g), g.shape[0], _ptr(out), ctypes.byref(n))
+    if rc != 0:
+        raise OracleError(rc)
+    return out, int(n.value)
+
+
+def phase_window(slice_bytes: int, sm_reach_bytes: int, max_parts: int = 64):
+    """(parts, sub_bytes) of the moving sub-windows."""
+    parts = ctypes.c_uint32()
+    sub = ctypes.c_uint64()
+    rc = _load().orc_phase_window(slice_bytes, sm_reach_bytes, max_parts, ctypes.byref(parts),
+                                  ctypes.byref(sub))
+    if rc != 0:
+        raise OracleError(rc)
+    return int(parts.value), int(sub.value)
+
+
+def rebalance_weights(work, finish_ns, scale: int = 1_000_000) -> np.ndarray:
+    w = np.ascontiguousarray(work, dtype=np.uint32)
+    f = np.ascontiguousarray(finish_ns, dtype=np.uint64)
+    if w.shape != f.shape:
+        raise OracleError(-1)
+    out = np.zeros(w.shape[0], dtype=np.uint32)
+    rc = _load().orc_rebalance_weights(_ptr(w), _ptr(f), w.shape[0], scale, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def group_finish(t_start, t_end, group_of_sm, n_groups: int):
+    """(finish_ns uint64[n_groups], span_ns) from the per-SM block timers of one run."""
+    a = np.ascontiguousarray(t_start, dtype=np.uint64)
+    b = np.ascontiguousarray(t_end, dtype=np.uint64)
+    g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+    out = np.zeros(n_groups, dtype=np.uint64)
+    span = ctypes.c_uint64()
+    rc = _load().orc_group_finish(_ptr(a), _ptr(b), _ptr(g), g.shape[0], n_groups, _ptr(out),
+                                  ctypes.byref(span))
+    if rc != 0:
+        raise OracleError(rc)
+    return out, int(span.value)
+
+
+def finish_spread_ppm(finish_ns) -> int:
+    f = np.ascontiguousarray(finish_ns, dtype=np.uint64)
+    ppm = ctypes.c_uint32()
+    rc = _load().orc_finish_spread_ppm(_ptr(f), f.shape[0], ctypes.byref(ppm))
+    if rc != 0:
+        raise OracleError(rc)
+    return int(ppm.value)
+
+
+def window_cover(windows, n_lines: int):
+    """(covered lines, smallest depth, largest depth) of a set of windows."""
+    w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+    wb = np.ascontiguousarray(w[:, 0])
+    wn = np.ascontiguousarray(w[:, 1])
+    cov = ctypes.c_uint64()
+    lo = ctypes.c_uint32()
+    hi = ctypes.c_uint32()
+    rc = _load().orc_window_cover(_ptr(wb), _ptr(wn), w.shape[0], n_lines, ctypes.byref(cov),
+                                  ctypes.byref(lo), ctypes.byref(hi))
+    if rc != 0:
+        raise OracleError(rc)
+    return int(cov.value), int(lo.value), int(hi.value)
+
+
+def probe_rate(t_start, t_end, claim, solo: bool, total_reads: int):
+    """(GB/s, seconds, overlap) of one probe from its timers; OracleError(-6) if an SM never ran."""
+    a = np.ascontiguousarray(t_start, dtype=np.uint64)
+    b = np.ascontiguousarray(t_end, dtype=np.uint64)
+    c = np.ascontiguousarray(claim, dtype=np.uint32)
+    g = ctypes.c_double()
+    sec = ctypes.c_double()
+    ov = ctypes.c_double()
+    rc = _load().orc_probe_rate(_ptr(a), _ptr(b), _ptr(c), 1 if solo else 0, total_reads,
+                                ctypes.byref(g), ctypes.byref(sec), ctypes.byref(ov))
+    if rc != 0:
+        raise OracleError(rc)
+    return float(g.value), float(sec.value), float(ov.value)
 
 
 def n_threads() -> int:

@@ -7,8 +7,8 @@
  *
  * What it defines (the paper gives prose only, so every definition below is a
  * stated reading of that prose):
- *   - Section 2.1 "Basic benchmark": every warp reads random coalesced arrays of
- *     32 words (32-, 64- or 128-bit) inside a memory region; here the region has
+ *   - Section 2.1 (the basic benchmark): each warp fetches whole lines of 32 words
+ *     (32-, 64- or 128-bit) at random positions inside a memory region; here the region has
  *     known contents (a hash of the word index), the random line comes from a
  *     counter-based generator, and what is read is folded into two checksums per
  *     warp so that a reader can prove which lines were touched.
@@ -124,8 +124,8 @@ void orc_warp_checksum(uint32_t index_mode, uint64_t seed, uint64_t v, uint64_t 
 }
 
 /* ---- O3b: windows that move with time ------------------------------------------
- * Section 1.3 asks that "any particular warp only accesses a smaller region"; the
- * paper fixes that region for good.  Reading for hardware whose per-SM translation
+ * Section 1.3 wants each warp confined to a part of memory smaller than the reach; the
+ * paper fixes that part for good.  Reading for hardware whose per-SM translation
  * cache is smaller than its share of memory: the warp's window of n lines is cut into
  * Q = ceil(n / sub_lines) sub-windows [floor(n q / Q), floor(n (q+1) / Q)); reads come
  * in phases of phase_reads reads, phase p = floor(i / phase_reads) of a warp's stream
@@ -164,6 +164,77 @@ void orc_warp_checksum_phased(uint64_t seed, uint64_t v, uint64_t first_read, ui
 }
 
 static int orc_width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
+
+/* ---- O3c: a stream that mixes sequential and random reads ----------------------------
+ * Section 2.1 ends by noting that sequential access runs faster than random access; a real
+ * workload is often a blend.  Reading: with a period k >= 1, read i of a warp's stream is
+ * sequential when i mod k == 0 -- it is read number i/k of the warp's sequential walk,
+ * line = base + ((i/k) * n_warps_total + v) mod n, exactly the STRIDE rule applied to the
+ * counter i/k -- and random otherwise (the RANDOM rule at the same i).  k = 1 is the
+ * sequential mode; as k grows the stream tends to the random mode.                     */
+uint64_t orc_line_mixed(uint64_t seed, uint64_t v, uint64_t n_warps_total, uint64_t i,
+                        uint64_t base, uint64_t n, uint64_t mix_period)
+{
+    if (i % mix_period == 0)
+        return orc_line(ORC_INDEX_STRIDE, seed, v, n_warps_total, i / mix_period, base, n);
+    return orc_line(ORC_INDEX_RANDOM, seed, v, n_warps_total, i, base, n);
+}
+
+void orc_warp_checksum_mixed(uint64_t seed, uint64_t v, uint64_t n_warps_total, uint64_t first_read,
+                             uint64_t reads, uint32_t W, uint64_t base, uint64_t n,
+                             uint64_t mix_period, uint32_t *X, uint32_t *S)
+{
+    uint32_t x = 0, s = 0;
+    for (uint64_t t = 0; t < reads; ++t) {
+        uint64_t line = orc_line_mixed(seed, v, n_warps_total, first_read + t, base, n, mix_period);
+        for (uint32_t lane = 0; lane < 32; ++lane)
+            for (uint32_t w = 0; w < W; ++w) {
+                uint32_t word = orc_word(line * 32u * W + (uint64_t)lane * W + w);
+                x ^= word;
+                s += word;
+            }
+    }
+    *X = x;
+    *S = s;
+}
+
+/* Per-SM mode with the mixed stream; arguments as orc_read_per_sm.                      */
+int32_t orc_read_per_sm_mixed(uint64_t region_bytes, uint32_t W, uint32_t nsm, uint32_t wps,
+                              uint64_t first_read, uint64_t reads, uint64_t seed,
+                              const uint16_t *group_of_sm, const uint32_t *win_base,
+                              const uint32_t *win_n, uint32_t n_groups, uint64_t mix_period,
+                              uint32_t *out)
+{
+    if (!orc_width_ok(W) || !out || nsm == 0 || wps == 0 || mix_period == 0) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    if (group_of_sm) {
+        if (!win_base || !win_n || n_groups == 0) return ORC_ERR_ARG;
+        for (uint32_t g = 0; g < n_groups; ++g)
+            if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
+        for (uint32_t s = 0; s < nsm; ++s)
+            if (group_of_sm[s] != ORC_SM_INACTIVE && group_of_sm[s] >= n_groups) return ORC_ERR_MAP;
+    }
+    uint64_t total = (uint64_t)nsm * wps;
+    int64_t nw = (int64_t)total;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t sm = (uint32_t)(v / wps);
+        uint64_t base = 0, n = L;
+        if (group_of_sm) {
+            if (group_of_sm[sm] == ORC_SM_INACTIVE) {
+                out[2 * v] = 0;
+                out[2 * v + 1] = 0;
+                continue;
+            }
+            base = win_base[group_of_sm[sm]];
+            n = win_n[group_of_sm[sm]];
+        }
+        orc_warp_checksum_mixed(seed, (uint64_t)v, total, first_read, reads, W, base, n, mix_period,
+                                &out[2 * v], &out[2 * v + 1]);
+    }
+    return ORC_OK;
+}
 
 /* Per-SM mode with moving windows (see orc_line_phased); arguments as orc_read_per_sm.
  * nsm = 0 with group_of_sm = NULL is not accepted; for logical warps over the whole
@@ -293,22 +364,42 @@ int32_t orc_read_per_sm(uint64_t region_bytes, uint32_t W, uint32_t index_mode,
     return ORC_OK;
 }
 
-/* ---- O4: windows (Section 1.3 "half the memory for simplicity", Section 2.4) ---
+/* ---- O4: windows (Section 1.3: a window below the reach, half the memory as the simple
+ * case; Section 2.4) ---------------------------------------------------------------
  * L lines are cut into K = ceil(L / S_lines) chunks of floor(L/K) lines, the last
  * one running to L.  policy 0: group g takes chunk g mod K.  policy 1 (the
  * paper's naive control, one "group" per SM): chunk sm64(seed ^ g) mod K.
- * coverage = distinct chunks used / K.                                          */
+ * coverage = distinct chunks used / K.
+ * policy 2 (Section 1.3 only asks that each warp's window stay below the reach; the
+ * windows need not be disjoint): G windows of exactly S_lines lines, evenly spaced with
+ * overlap, base_g = floor(g * (L - S_lines) / (G - 1)) (base 0 when G = 1), so the first
+ * starts at line 0 and the last ends at line L.  coverage = lines inside at least one
+ * window / L, which is 1 exactly when no step between bases exceeds S_lines.           */
 int32_t orc_make_windows(uint64_t region_bytes, uint32_t W, uint64_t window_bytes,
                          uint32_t n_groups, uint32_t policy, uint64_t seed,
                          uint32_t *win_base, uint32_t *win_n, double *coverage)
 {
-    if (!orc_width_ok(W) || n_groups == 0 || policy > 1 || !win_base || !win_n) return ORC_ERR_ARG;
+    if (!orc_width_ok(W) || n_groups == 0 || policy > 2 || !win_base || !win_n) return ORC_ERR_ARG;
     uint64_t line_bytes = 128ull * W;
     uint64_t L = region_bytes / line_bytes;
     if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
     uint64_t S = window_bytes / line_bytes;
     if (S < 1) S = 1;
     if (S > L) S = L;
+    if (policy == 2) {
+        uint64_t covered = 0, end_prev = 0;
+        for (uint32_t g = 0; g < n_groups; ++g) {
+            uint64_t base = n_groups > 1 ? (uint64_t)g * (L - S) / (n_groups - 1) : 0;
+            win_base[g] = (uint32_t)base;
+            win_n[g] = (uint32_t)S;
+            /* bases do not decrease: lines newly covered by this window */
+            uint64_t from = base > end_prev ? base : end_prev;
+            if (base + S > from) covered += base + S - from;
+            if (base + S > end_prev) end_prev = base + S;
+        }
+        if (coverage) *coverage = (double)covered / (double)L;
+        return ORC_OK;
+    }
     uint64_t K = (L + S - 1) / S;
     uint64_t chunk = L / K;
     unsigned char *used = (unsigned char *)calloc((size_t)K, 1);
@@ -325,6 +416,56 @@ int32_t orc_make_windows(uint64_t region_bytes, uint32_t W, uint64_t window_byte
     for (uint64_t c = 0; c < K; ++c) distinct += used[c];
     free(used);
     if (coverage) *coverage = (double)distinct / (double)K;
+    return ORC_OK;
+}
+
+/* How evenly a set of windows covers the region: for every line, depth = number of
+ * windows that contain it.  With equal work per window and equal window sizes the read
+ * density at a line is proportional to its depth.  Returns the number of lines with
+ * depth >= 1 and the smallest and largest depth over those lines (plain sweep over the
+ * 2G window edges).                                                                   */
+int32_t orc_window_cover(const uint32_t *win_base, const uint32_t *win_n, uint32_t n_groups,
+                         uint64_t n_lines, uint64_t *covered, uint32_t *depth_min,
+                         uint32_t *depth_max)
+{
+    if (!win_base || !win_n || !covered || !depth_min || !depth_max || n_groups == 0)
+        return ORC_ERR_ARG;
+    for (uint32_t g = 0; g < n_groups; ++g)
+        if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > n_lines) return ORC_ERR_RANGE;
+    uint64_t *edge = (uint64_t *)malloc(sizeof(uint64_t) * 2 * n_groups);
+    if (!edge) return ORC_ERR_ARG;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        edge[2 * g] = win_base[g];
+        edge[2 * g + 1] = (uint64_t)win_base[g] + win_n[g];
+    }
+    /* insertion sort of the distinct edge positions: G <= a few hundred */
+    uint32_t ne = 2 * n_groups;
+    for (uint32_t i = 1; i < ne; ++i) {
+        uint64_t x = edge[i];
+        uint32_t j = i;
+        while (j > 0 && edge[j - 1] > x) {
+            edge[j] = edge[j - 1];
+            --j;
+        }
+        edge[j] = x;
+    }
+    uint64_t cov = 0;
+    uint32_t dmin = 0xFFFFFFFFu, dmax = 0;
+    for (uint32_t i = 0; i + 1 < ne; ++i) {
+        uint64_t a = edge[i], b = edge[i + 1];
+        if (b == a) continue;
+        uint32_t depth = 0; /* windows containing the stretch [a, b) */
+        for (uint32_t g = 0; g < n_groups; ++g)
+            if (win_base[g] <= a && b <= (uint64_t)win_base[g] + win_n[g]) ++depth;
+        if (depth == 0) continue;
+        cov += b - a;
+        if (depth < dmin) dmin = depth;
+        if (depth > dmax) dmax = depth;
+    }
+    free(edge);
+    *covered = cov;
+    *depth_min = dmin == 0xFFFFFFFFu ? 0 : dmin;
+    *depth_max = dmax;
     return ORC_OK;
 }
 
@@ -572,7 +713,7 @@ int32_t orc_cluster(const float *T, uint32_t n, uint32_t flags, int32_t *group_o
         double sigma = (1.4826 * mad) / sqrt((double)merge_pairs[best_k]);
         double conf = sigma > 0.0 ? best_gap / sigma : (best_gap > 0.0 ? INFINITY : 0.0);
         if (confidence) *confidence = conf;
-        /* the paper sets the "more faint pattern in the background" aside (Section 2.2):
+        /* Section 2.2 sets the fainter background structure of its matrix aside:
          * a gap below 1 % of the median pair rate (2^20 in these units) is no group boundary */
         if (!(best_gap >= 4.0 * sigma) || !(best_gap >= 10485.76)) goto done; /* one group */
         /* 6. canonical labels: representatives are smallest members */
@@ -637,4 +778,234 @@ int32_t orc_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_poi
     for (uint32_t k = 0; k < first_bad; ++k)
         if (gbps[k] >= 0.9 * P) *reach_bytes = size_bytes[k];
     return cliff;
+}
+
+/* ---- O6b: next size to measure when refining the reach ---------------------------
+ * The sweep of Section 2.1 / Fig. 1 only brackets the cliff between two of its sizes.
+ * Reading: bisect between the reach found so far (good) and the smallest measured size
+ * above it (bad) on a grid of `step` bytes: mid = floor((good + bad) / 2 / step) * step.
+ * Returns 1 and *next_size = mid while bad - good > step and good < mid < bad; 0 when
+ * the refinement is finished or the sweep shows no cliff.  A measured point is judged by
+ * orc_reach itself (it is appended to the sweep and the rule is applied again), so there
+ * is no second acceptance threshold.                                                 */
+int32_t orc_reach_next(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
+                       uint64_t step_bytes, uint64_t *next_size)
+{
+    if (!next_size || step_bytes == 0) return ORC_ERR_ARG;
+    double plateau;
+    uint64_t good;
+    int32_t rc = orc_reach(size_bytes, gbps, n_points, &plateau, &good);
+    if (rc < 0) return rc;
+    *next_size = 0;
+    if (rc == 0) return 0;
+    uint64_t bad = 0;
+    for (uint32_t k = 0; k < n_points; ++k)
+        if (size_bytes[k] > good) {
+            bad = size_bytes[k];
+            break; /* sizes increase: the first one above is the smallest */
+        }
+    if (bad == 0 || bad - good <= step_bytes) return 0;
+    uint64_t mid = (good + bad) / 2 / step_bytes * step_bytes;
+    if (mid <= good || mid >= bad) return 0;
+    *next_size = mid;
+    return 1;
+}
+
+/* ---- O7: how far one SM's own translation cache reaches ------------------------------
+ * Same experiment as Section 2.1 with one window per SM: rate versus window size, sizes
+ * increasing.  Reading: the level the small windows sustain is the middle one of the
+ * first three rates (the only rate if fewer than three points); the reach is the last
+ * size of the leading run of points whose rate is at least keep * that level.  A sweep
+ * whose very first point already falls short returns its first size.                  */
+int32_t orc_sm_reach(const uint64_t *size_bytes, const double *gbps, uint32_t n_points,
+                     double keep, uint64_t *reach_bytes)
+{
+    if (!size_bytes || !gbps || !reach_bytes || n_points == 0 || !(keep > 0.0) || keep > 1.0)
+        return ORC_ERR_ARG;
+    for (uint32_t k = 1; k < n_points; ++k)
+        if (size_bytes[k] <= size_bytes[k - 1]) return ORC_ERR_ARG;
+    double top;
+    if (n_points >= 3) {
+        double a = gbps[0], b = gbps[1], c = gbps[2];
+        /* middle of three */
+        if ((a <= b && b <= c) || (c <= b && b <= a)) top = b;
+        else if ((b <= a && a <= c) || (c <= a && a <= b)) top = a;
+        else top = c;
+    } else {
+        top = gbps[0];
+    }
+    *reach_bytes = size_bytes[0];
+    for (uint32_t k = 0; k < n_points; ++k) {
+        if (gbps[k] >= keep * top) *reach_bytes = size_bytes[k];
+        else break;
+    }
+    return ORC_OK;
+}
+
+/* ---- O8: one window per SM, the SMs of a resource group side by side -----------------
+ * Section 2.4 gives every group one chunk.  A finer reading that still keeps every group
+ * below its reach: every active SM gets a window id of its own, ids handed out group by
+ * group (groups in increasing number, SMs of a group in increasing SM id), so that with
+ * windows laid out in id order the windows of one group's SMs are neighbours and together
+ * form the group's chunk.  Inactive SMs (0xFFFF) stay inactive.  Returns the number of ids. */
+int32_t orc_owner_map(const uint16_t *group_of_sm, uint32_t nsm, uint16_t *owner_of_sm,
+                      uint32_t *n_owners)
+{
+    if (!group_of_sm || !owner_of_sm || !n_owners || nsm == 0 || nsm > 65535u) return ORC_ERR_ARG;
+    uint32_t next = 0;
+    uint32_t max_g = 0;
+    int any = 0;
+    for (uint32_t s = 0; s < nsm; ++s)
+        if (group_of_sm[s] != ORC_SM_INACTIVE) {
+            if (!any || group_of_sm[s] > max_g) max_g = group_of_sm[s];
+            any = 1;
+        }
+    for (uint32_t s = 0; s < nsm; ++s) owner_of_sm[s] = ORC_SM_INACTIVE;
+    if (any)
+        for (uint32_t g = 0; g <= max_g; ++g)
+            for (uint32_t s = 0; s < nsm; ++s)
+                if (group_of_sm[s] == g) owner_of_sm[s] = (uint16_t)next++;
+    *n_owners = next;
+    return ORC_OK;
+}
+
+/* ---- O9: size of the moving sub-windows (see orc_line_phased) ---------------------------
+ * Two phases of a warp's stream can be live at once, and the SM's translation cache
+ * should hold both with room to spare: the slice an SM works through is cut into the
+ * smallest power-of-two number of parts (at most max_parts) that makes a part no larger
+ * than a quarter of the SM's reach; sub = ceil(slice / parts).                        */
+int32_t orc_phase_window(uint64_t slice_bytes, uint64_t sm_reach_bytes, uint32_t max_parts,
+                         uint32_t *parts, uint64_t *sub_bytes)
+{
+    if (!parts || !sub_bytes || slice_bytes == 0 || sm_reach_bytes == 0 || max_parts == 0)
+        return ORC_ERR_ARG;
+    uint32_t q = 1;
+    /* slice / q > reach / 4   <=>   4 * slice > reach * q   (exact in integers) */
+    while (q < max_parts && (unsigned __int128)4 * slice_bytes > (unsigned __int128)sm_reach_bytes * q)
+        q *= 2;
+    *parts = q;
+    *sub_bytes = (slice_bytes + q - 1) / q;
+    return ORC_OK;
+}
+
+/* ---- O10: new capacity weights from one observed run -----------------------------------
+ * Section 2.3: a group's throughput belongs to the group.  After a run in which group g
+ * did work[g] units and its last SM finished finish_ns[g] after the common start, the
+ * group has shown the rate work/finish.  Reading, in integers so that nothing depends on
+ * rounding mode: rate_g = max(1, floor(work_g * 2^48 / finish_g)); a group that was not
+ * seen (finish 0 or no work) keeps a token rate of max(1, smallest seen rate / 1024); the
+ * new weight is the rate's share of `scale`, rounded half up, at least 1:
+ *   w_g = max(1, floor((rate_g * scale + total / 2) / total)),  total = sum of rates.
+ * At a fixed point (every group finishing together) the weights reproduce the work
+ * shares.  (work < 2^32, scale < 2^32: every product stays below 2^128.)              */
+int32_t orc_rebalance_weights(const uint32_t *work, const uint64_t *finish_ns, uint32_t n_groups,
+                              uint32_t scale, uint32_t *weight)
+{
+    typedef unsigned __int128 u128;
+    if (!work || !finish_ns || !weight || n_groups == 0 || scale == 0) return ORC_ERR_ARG;
+    u128 *rate = (u128 *)malloc(sizeof(u128) * n_groups);
+    if (!rate) return ORC_ERR_ARG;
+    u128 slowest = 0;
+    int seen = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        rate[g] = 0;
+        if (finish_ns[g] == 0 || work[g] == 0) continue;
+        rate[g] = ((u128)work[g] << 48) / finish_ns[g];
+        if (rate[g] == 0) rate[g] = 1;
+        if (!seen || rate[g] < slowest) slowest = rate[g];
+        seen = 1;
+    }
+    if (!seen) {
+        free(rate);
+        return ORC_ERR_RANGE; /* no group finished any work */
+    }
+    u128 token = slowest / 1024;
+    if (token == 0) token = 1;
+    u128 total = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        if (rate[g] == 0) rate[g] = token;
+        total += rate[g];
+    }
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        u128 w = (rate[g] * scale + total / 2) / total;
+        weight[g] = w == 0 ? 1u : (uint32_t)w;
+    }
+    free(rate);
+    return ORC_OK;
+}
+
+/* When each group finished, from the per-SM block timers of one run (ns; t_end = 0 for an
+ * SM that ran no block): the common start is the earliest start over the SMs that ran,
+ * finish[g] = latest end over group g's SMs that ran, minus that start (at least 1; 0 if
+ * none of the group's SMs ran); *span = latest end overall minus the common start.    */
+int32_t orc_group_finish(const uint64_t *t_start, const uint64_t *t_end, const uint16_t *group_of_sm,
+                         uint32_t nsm, uint32_t n_groups, uint64_t *finish_ns, uint64_t *span_ns)
+{
+    if (!t_start || !t_end || !group_of_sm || !finish_ns || !span_ns || nsm == 0 || n_groups == 0)
+        return ORC_ERR_ARG;
+    uint64_t begin = 0, last = 0;
+    int any = 0;
+    for (uint32_t s = 0; s < nsm; ++s) {
+        if (t_end[s] == 0) continue;
+        if (!any || t_start[s] < begin) begin = t_start[s];
+        if (!any || t_end[s] > last) last = t_end[s];
+        any = 1;
+    }
+    for (uint32_t g = 0; g < n_groups; ++g) finish_ns[g] = 0;
+    *span_ns = any ? last - begin : 0;
+    for (uint32_t s = 0; s < nsm; ++s) {
+        if (t_end[s] == 0 || group_of_sm[s] == ORC_SM_INACTIVE) continue;
+        if (group_of_sm[s] >= n_groups) return ORC_ERR_MAP;
+        uint64_t f = t_end[s] > begin ? t_end[s] - begin : 1;
+        if (f > finish_ns[group_of_sm[s]]) finish_ns[group_of_sm[s]] = f;
+    }
+    return ORC_OK;
+}
+
+/* (latest - earliest) / latest over the groups that ran, in parts per million, rounded
+ * down: how far from finishing together the groups of a balanced run were.            */
+int32_t orc_finish_spread_ppm(const uint64_t *finish_ns, uint32_t n_groups, uint32_t *ppm)
+{
+    if (!finish_ns || !ppm || n_groups == 0) return ORC_ERR_ARG;
+    uint64_t lo = 0, hi = 0;
+    int seen = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        if (finish_ns[g] == 0) continue;
+        if (!seen || finish_ns[g] < lo) lo = finish_ns[g];
+        if (!seen || finish_ns[g] > hi) hi = finish_ns[g];
+        seen = 1;
+    }
+    *ppm = seen ? (uint32_t)(((unsigned __int128)(hi - lo) * 1000000u) / hi) : 0u;
+    return ORC_OK;
+}
+
+/* ---- O11: rate and overlap of one two-SM probe (Section 2.2, Fig. 2) --------------------
+ * Each chosen SM performs total_reads / 2 line reads of 128 bytes.  The pair's throughput
+ * counts the bytes of both SMs over the union of their two intervals,
+ *   GB/s = bytes / (latest end - earliest start)        (timers in ns, so bytes/ns = GB/s)
+ * and the figure only means contention if the two ran side by side:
+ *   overlap = (earliest end - latest start) / (latest end - earliest start), 0 if disjoint.
+ * A solo run (one SM) has overlap 1.  An SM that claimed nothing or never ended: -6.     */
+#define ORC_ERR_SM_UNCOVERED (-6)
+int32_t orc_probe_rate(const uint64_t *t_start, const uint64_t *t_end, const uint32_t *claim,
+                       uint32_t solo, uint64_t total_reads, double *gbps, double *seconds,
+                       double *overlap)
+{
+    if (!t_start || !t_end || !claim || !gbps || !seconds || !overlap || solo > 1) return ORC_ERR_ARG;
+    uint32_t k = solo ? 1 : 2;
+    for (uint32_t i = 0; i < k; ++i)
+        if (claim[i] == 0 || t_end[i] == 0 || t_end[i] < t_start[i]) return ORC_ERR_SM_UNCOVERED;
+    uint64_t s_lo = t_start[0], s_hi = t_start[0], e_lo = t_end[0], e_hi = t_end[0];
+    if (k == 2) {
+        if (t_start[1] < s_lo) s_lo = t_start[1];
+        if (t_start[1] > s_hi) s_hi = t_start[1];
+        if (t_end[1] < e_lo) e_lo = t_end[1];
+        if (t_end[1] > e_hi) e_hi = t_end[1];
+    }
+    uint64_t span = e_hi - s_lo;
+    uint64_t bytes = (total_reads / 2) * k * 128ull;
+    *seconds = (double)span * 1e-9;
+    *gbps = span ? (double)bytes / (double)span : 0.0;
+    *overlap = (span && e_lo > s_hi) ? (double)(e_lo - s_hi) / (double)span : 0.0;
+    return ORC_OK;
 }

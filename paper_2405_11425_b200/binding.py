@@ -22,16 +22,18 @@ RR_ERR_STATIC_LIMIT = -10
 RR_STATIC_MAX_SM, RR_STATIC_SCRATCH_BYTES = 192, 5888
 RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0xFFFF
 RR_MODE_LOGICAL, RR_MODE_PER_SM, RR_MODE_POOLED = 0, 1, 2
-RR_INDEX_RANDOM, RR_INDEX_STRIDE, RR_INDEX_PHASED = 0, 1, 2
+RR_INDEX_RANDOM, RR_INDEX_STRIDE, RR_INDEX_PHASED, RR_INDEX_MIXED = 0, 1, 2, 3
 RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED, RR_VARIANT_PACKED = 0, 1, 2
-RR_VARIANT_L2_128, RR_VARIANT_L2_256, RR_VARIANT_BULK = 3, 4, 5
+RR_VARIANT_L2_128, RR_VARIANT_L2_256, RR_VARIANT_BULK, RR_VARIANT_SORTED = 3, 4, 5, 6
 
 EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
     "rr_random_read", "rr_read_report", "rr_probe_pair", "rr_probe_matrix_scratch_bytes",
     "rr_probe_matrix", "rr_cluster", "rr_make_windows", "rr_reach", "rr_random_read_static",
     "rr_gpc_map", "rr_make_weighted_windows",
-    "rr_read_block_times", "rr_host_counters",
+    "rr_read_block_times", "rr_host_counters", "rr_probe_rate", "rr_reach_next", "rr_sm_reach",
+    "rr_owner_map", "rr_phase_window", "rr_rebalance_weights", "rr_finish_spread_ppm",
+    "rr_window_cover", "rr_group_finish", "rr_probe_rows",
 )
 
 
@@ -60,8 +62,9 @@ class _ReadParams(ctypes.Structure):
         ("windows", ctypes.c_void_p), ("n_groups", ctypes.c_uint32),
         ("variant", ctypes.c_uint32), ("unroll", ctypes.c_uint32),
         ("pool_block_reads", ctypes.c_uint32), ("warp_start", ctypes.c_void_p),
-        ("phase_reads", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("phase_reads", ctypes.c_uint32), ("mix_period", ctypes.c_uint32),
         ("phase_window_bytes", ctypes.c_uint64),
+        ("sort_parts", ctypes.c_uint32), ("sort_reads", ctypes.c_uint32),
     ]
 
 
@@ -120,7 +123,7 @@ def _load():
     lib.rr_last_cuda_error.restype = ctypes.c_char_p
     lib.rr_last_cuda_error.argtypes = []
     lib.rr_device_info.restype = i32
-    lib.rr_device_info.argtypes = [p]
+    lib.rr_device_info.argtypes = [p, p, p]
     lib.rr_scratch_bytes.restype = ctypes.c_size_t
     lib.rr_scratch_bytes.argtypes = []
     lib.rr_fill.restype = i32
@@ -138,7 +141,27 @@ def _load():
     lib.rr_probe_matrix_scratch_bytes.restype = ctypes.c_size_t
     lib.rr_probe_matrix_scratch_bytes.argtypes = [u32]
     lib.rr_probe_matrix.restype = i32
-    lib.rr_probe_matrix.argtypes = [p, u64, u64, u32, u64, u32, p, u32, p, p, p, p]
+    lib.rr_probe_matrix.argtypes = [p, u64, u64, u32, u64, u32, p, u32, p, p, p, p, p]
+    lib.rr_probe_rows.restype = i32
+    lib.rr_probe_rows.argtypes = [p, u64, u64, u32, u64, u32, u32, u32, p, u32, p, p, p, p, p]
+    lib.rr_probe_rate.restype = i32
+    lib.rr_probe_rate.argtypes = [p, p, p, u32, u64, p, p, p]
+    lib.rr_reach_next.restype = i32
+    lib.rr_reach_next.argtypes = [p, p, u32, u64, p]
+    lib.rr_sm_reach.restype = i32
+    lib.rr_sm_reach.argtypes = [p, p, u32, d, p]
+    lib.rr_owner_map.restype = i32
+    lib.rr_owner_map.argtypes = [p, u32, p, p]
+    lib.rr_phase_window.restype = i32
+    lib.rr_phase_window.argtypes = [u64, u64, u32, p, p]
+    lib.rr_rebalance_weights.restype = i32
+    lib.rr_rebalance_weights.argtypes = [p, p, u32, u32, p]
+    lib.rr_group_finish.restype = i32
+    lib.rr_group_finish.argtypes = [p, p, p, u32, u32, p, p]
+    lib.rr_finish_spread_ppm.restype = i32
+    lib.rr_finish_spread_ppm.argtypes = [p, u32, p]
+    lib.rr_window_cover.restype = i32
+    lib.rr_window_cover.argtypes = [p, u32, u64, p, p, p]
     lib.rr_cluster.restype = i32
     lib.rr_cluster.argtypes = [p, u32, u32, p, p, p, p, p, p]
     lib.rr_gpc_map.restype = i32
@@ -182,9 +205,12 @@ def rr_strerror(code: int) -> str:
     return _load().rr_strerror(code).decode()
 
 
-def rr_device_info() -> dict:
+def rr_device_info(scratch=None, stream=None) -> dict:
+    """Facts of the current device; nsm_reg (%nsmid) is read only when a scratch buffer is given."""
     info = _DeviceInfo()
-    _check(_load().rr_device_info(ctypes.byref(info)), "rr_device_info")
+    _check(_load().rr_device_info(ctypes.byref(info), _dev(scratch),
+                                  _stream(stream) if scratch is not None else None),
+           "rr_device_info")
     out = {k: getattr(info, k) for k, _ in _DeviceInfo._fields_}
     out["name"] = info.name.decode()
     out["uuid"] = info.uuid.decode()
@@ -219,7 +245,8 @@ class ReadParams:
                  nsm: int = 0, reads_per_warp: int = 0, first_read: int = 0, seed: int = 0,
                  group_of_sm=None, windows=None, variant: int = RR_VARIANT_LDG, unroll: int = 0,
                  warp_start=None, pool_block_reads: int = 0, phase_reads: int = 0,
-                 phase_window_bytes: int = 0):
+                 phase_window_bytes: int = 0, mix_period: int = 0, sort_parts: int = 0,
+                 sort_reads: int = 0):
         self._groups = None
         self._windows = None
         self._warp_start = None
@@ -239,7 +266,7 @@ class ReadParams:
             self._windows.ctypes.data if self._windows is not None else None,
             n_groups, variant, unroll, pool_block_reads,
             self._warp_start.ctypes.data if self._warp_start is not None else None,
-            phase_reads, 0, phase_window_bytes)
+            phase_reads, mix_period, phase_window_bytes, sort_parts, sort_reads)
 
 
 def _result(r: _Result) -> ReadResult:
@@ -293,15 +320,54 @@ def rr_probe_pair(buf, region_bytes: int, sm_a: int, sm_b: int, total_reads: int
     return _result(res)
 
 
+class _ProbeStats(ctypes.Structure):
+    _fields_ = [("overlap_min", ctypes.c_double), ("pairs_below_goal", ctypes.c_uint32),
+                ("reruns", ctypes.c_uint32), ("relaunched", ctypes.c_uint32)]
+
+
 def rr_probe_matrix(buf, region_bytes: int, total_reads: int, warps_per_sm: int, seed: int,
-                    repeats: int, nsm: int, out, scratch, stream=None):
-    """Returns (T float32[nsm,nsm], smallest pair-overlap fraction)."""
+                    repeats: int, nsm: int, out, scratch, stream=None, *, with_overlaps=False):
+    """Returns (T float32[nsm,nsm], stats dict) -- plus the per-pair overlap matrix if asked."""
     T = np.zeros((nsm, nsm), dtype=np.float32)
-    ov = ctypes.c_double()
+    ov = np.ones((nsm, nsm), dtype=np.float32) if with_overlaps else None
+    st = _ProbeStats()
     _check(_load().rr_probe_matrix(_dev(buf), region_bytes, total_reads, warps_per_sm, seed,
                                    repeats, T.ctypes.data, nsm, _dev(out), _dev(scratch),
-                                   ctypes.byref(ov), _stream(stream)), "rr_probe_matrix")
-    return T, float(ov.value)
+                                   ctypes.byref(st), ov.ctypes.data if with_overlaps else None,
+                                   _stream(stream)), "rr_probe_matrix")
+    stats = {"overlap_min": float(st.overlap_min), "pairs_below_goal": int(st.pairs_below_goal),
+             "reruns": int(st.reruns), "relaunched": int(st.relaunched)}
+    return (T, stats, ov) if with_overlaps else (T, stats)
+
+
+def rr_probe_rows(buf, region_bytes: int, total_reads: int, warps_per_sm: int, seed: int,
+                  repeats: int, row_begin: int, row_end: int, T, out, scratch, overlaps=None,
+                  stream=None) -> dict:
+    """Probes rows [row_begin, row_end) into the caller's matrix T (float32 [nsm, nsm], updated
+    in place; `overlaps` likewise if given).  Returns the stats of these rows."""
+    if T.dtype != np.float32 or T.ndim != 2 or T.shape[0] != T.shape[1] or \
+            not T.flags["C_CONTIGUOUS"]:
+        raise RRError(RR_ERR_ARG, "rr_probe_rows")
+    st = _ProbeStats()
+    _check(_load().rr_probe_rows(_dev(buf), region_bytes, total_reads, warps_per_sm, seed, repeats,
+                                 row_begin, row_end, T.ctypes.data, T.shape[0], _dev(out),
+                                 _dev(scratch), ctypes.byref(st),
+                                 overlaps.ctypes.data if overlaps is not None else None,
+                                 _stream(stream)), "rr_probe_rows")
+    return {"overlap_min": float(st.overlap_min), "pairs_below_goal": int(st.pairs_below_goal),
+            "reruns": int(st.reruns), "relaunched": int(st.relaunched)}
+
+
+def rr_probe_rate(t_start, t_end, claim, solo: bool, total_reads: int):
+    """(GB/s, seconds, overlap) of one probe from its timers (host rule, no GPU involved)."""
+    a = np.ascontiguousarray(t_start, dtype=np.uint64)
+    b = np.ascontiguousarray(t_end, dtype=np.uint64)
+    c = np.ascontiguousarray(claim, dtype=np.uint32)
+    g, sec, ov = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    _check(_load().rr_probe_rate(a.ctypes.data, b.ctypes.data, c.ctypes.data, 1 if solo else 0,
+                                 total_reads, ctypes.byref(g), ctypes.byref(sec), ctypes.byref(ov)),
+           "rr_probe_rate")
+    return float(g.value), float(sec.value), float(ov.value)
 
 
 RR_CLUSTER_SOLO_NORMALISE = 1
@@ -368,3 +434,90 @@ def rr_reach(size_bytes, gbps):
     if rc < 0:
         raise RRError(rc, "rr_reach")
     return bool(rc), float(plateau.value), int(r.value)
+
+
+def rr_reach_next(size_bytes, gbps, step_bytes: int) -> int:
+    """Next size to measure while refining the reach, or 0 when the refinement is finished."""
+    s = np.ascontiguousarray(size_bytes, dtype=np.uint64)
+    g = np.ascontiguousarray(gbps, dtype=np.float64)
+    if s.shape != g.shape or s.ndim != 1:
+        raise RRError(RR_ERR_ARG, "rr_reach_next")
+    nxt = ctypes.c_uint64()
+    rc = _load().rr_reach_next(s.ctypes.data, g.ctypes.data, len(s), step_bytes, ctypes.byref(nxt))
+    if rc < 0:
+        raise RRError(rc, "rr_reach_next")
+    return int(nxt.value) if rc else 0
+
+
+def rr_sm_reach(size_bytes, gbps, keep: float = 0.97) -> int:
+    s = np.ascontiguousarray(size_bytes, dtype=np.uint64)
+    g = np.ascontiguousarray(gbps, dtype=np.float64)
+    if s.shape != g.shape or s.ndim != 1:
+        raise RRError(RR_ERR_ARG, "rr_sm_reach")
+    r = ctypes.c_uint64()
+    _check(_load().rr_sm_reach(s.ctypes.data, g.ctypes.data, len(s), keep, ctypes.byref(r)),
+           "rr_sm_reach")
+    return int(r.value)
+
+
+def rr_owner_map(group_of_sm):
+    """(owner_of_sm uint16[nsm], n_owners): one window id per active SM, group by group."""
+    g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+    out = np.zeros(g.shape[0], dtype=np.uint16)
+    n = ctypes.c_uint32()
+    _check(_load().rr_owner_map(g.ctypes.data, g.shape[0], out.ctypes.data, ctypes.byref(n)),
+           "rr_owner_map")
+    return out, int(n.value)
+
+
+def rr_phase_window(slice_bytes: int, sm_reach_bytes: int, max_parts: int = 64):
+    """(parts, sub_bytes) of the moving sub-windows."""
+    parts = ctypes.c_uint32()
+    sub = ctypes.c_uint64()
+    _check(_load().rr_phase_window(slice_bytes, sm_reach_bytes, max_parts, ctypes.byref(parts),
+                                   ctypes.byref(sub)), "rr_phase_window")
+    return int(parts.value), int(sub.value)
+
+
+def rr_rebalance_weights(work, finish_ns, scale: int = 1_000_000) -> np.ndarray:
+    w = np.ascontiguousarray(work, dtype=np.uint32)
+    f = np.ascontiguousarray(finish_ns, dtype=np.uint64)
+    if w.shape != f.shape or w.ndim != 1:
+        raise RRError(RR_ERR_ARG, "rr_rebalance_weights")
+    out = np.zeros(w.shape[0], dtype=np.uint32)
+    _check(_load().rr_rebalance_weights(w.ctypes.data, f.ctypes.data, w.shape[0], scale,
+                                        out.ctypes.data), "rr_rebalance_weights")
+    return out
+
+
+def rr_group_finish(t_start, t_end, group_of_sm, n_groups: int):
+    """(finish_ns uint64[n_groups], span_ns) from the per-SM block timers of one run."""
+    a = np.ascontiguousarray(t_start, dtype=np.uint64)
+    b = np.ascontiguousarray(t_end, dtype=np.uint64)
+    g = np.ascontiguousarray(group_of_sm, dtype=np.uint16)
+    if not (a.shape == b.shape == g.shape) or a.ndim != 1:
+        raise RRError(RR_ERR_ARG, "rr_group_finish")
+    out = np.zeros(n_groups, dtype=np.uint64)
+    span = ctypes.c_uint64()
+    _check(_load().rr_group_finish(a.ctypes.data, b.ctypes.data, g.ctypes.data, g.shape[0],
+                                   n_groups, out.ctypes.data, ctypes.byref(span)),
+           "rr_group_finish")
+    return out, int(span.value)
+
+
+def rr_finish_spread_ppm(finish_ns) -> int:
+    f = np.ascontiguousarray(finish_ns, dtype=np.uint64)
+    ppm = ctypes.c_uint32()
+    _check(_load().rr_finish_spread_ppm(f.ctypes.data, f.shape[0], ctypes.byref(ppm)),
+           "rr_finish_spread_ppm")
+    return int(ppm.value)
+
+
+def rr_window_cover(windows, n_lines: int):
+    """(covered lines, smallest depth, largest depth) of a set of windows."""
+    w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+    cov = ctypes.c_uint64()
+    lo, hi = ctypes.c_uint32(), ctypes.c_uint32()
+    _check(_load().rr_window_cover(w.ctypes.data, w.shape[0], n_lines, ctypes.byref(cov),
+                                   ctypes.byref(lo), ctypes.byref(hi)), "rr_window_cover")
+    return int(cov.value), int(lo.value), int(hi.value)

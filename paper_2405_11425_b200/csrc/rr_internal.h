@@ -23,7 +23,8 @@ struct ProbeRecord {      // one per probe launch
     uint64_t t_start[2];
     uint64_t t_end[2];
     uint32_t claim[2];
-    uint32_t pad[2];
+    uint32_t ready;       // chosen SMs that have arrived at the common start
+    uint32_t gave_up;     // chosen SMs that stopped waiting for the other one
 };
 
 struct ScratchHeader {

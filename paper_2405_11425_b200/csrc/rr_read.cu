@@ -28,10 +28,24 @@ struct Tables {
 // How read i of a warp's stream picks its line inside the warp's window.
 struct IndexSpec {
     uint32_t mode;         // RR_INDEX_*
-    uint32_t phase_shift;  // PHASED: log2(reads per phase)
+    uint32_t phase_shift;  // PHASED: log2(reads per phase); MIXED: log2(mix period)
     uint32_t sub_lines;    // PHASED: largest sub-window, in lines
     uint32_t sm, nsm;      // PHASED, per-SM mode: this SM of nsm (nsm = 0: no stagger)
+    uint32_t sort_shift;   // SORTED variant: log2(parts of the window)
+    uint32_t sort_reads;   // SORTED variant: reads per part and epoch (a multiple of 32)
 };
+
+// The number read i of warp v reduces modulo its window length: a hash of (key, i) for a random
+// read, the walk counter for a sequential one (STRIDE: every read; MIXED: reads whose index is a
+// multiple of the period, which are read i/period of the warp's walk).
+__device__ __forceinline__ uint64_t draw_index(const IndexSpec &ix, uint64_t key, uint64_t i,
+                                               uint64_t v, uint64_t V)
+{
+    if (ix.mode == RR_INDEX_STRIDE) return i * V + v;
+    if (ix.mode == RR_INDEX_MIXED && !(i & ((1ull << ix.phase_shift) - 1)))
+        return (i >> ix.phase_shift) * V + v;
+    return sm64(key + i * kGamma);
+}
 
 // The window a batch of 32 reads draws from: the warp's whole window, or (PHASED) the
 // sub-window of the batch's phase.  Recomputed only when the phase changes.
@@ -83,7 +97,7 @@ struct ReadArgs {
 };
 
 constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarL2_128 = 3, kVarL2_256 = 4,
-              kVarBulk = 5;
+              kVarBulk = 5, kVarSorted = 6;
 __host__ __device__ constexpr int l2_hint_of(int var) { return var == kVarL2_128 ? 128 : (var == kVarL2_256 ? 256 : 0); }
 
 // Per-warp state of the bulk-copy shape: a ring of U line slots and U mbarriers in shared memory
@@ -91,7 +105,9 @@ __host__ __device__ constexpr int l2_hint_of(int var) { return var == kVarL2_128
 struct BulkRing {
     uint32_t ring, bars, phases;
     uint32_t *status;
+    uint32_t *queue;  // SORTED variant: this warp's ring of kSortQueue line indices (shared memory)
 };
+constexpr uint32_t kSortQueue = 64;  // two vectors of 32 lines
 constexpr uint32_t kBulkWaitPolls = 1u << 20;  // per line; each poll may itself sleep a little
 constexpr uint32_t kStatusBulkTimeout = 2u;    // status bit: a bulk copy did not complete in time
 
@@ -110,7 +126,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
     uint32_t x = 0, s = 0;
 
     auto gen = [&](uint64_t i) -> uint32_t {
-        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        const uint64_t r = draw_index(ix, key, i, v, V);
         return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[W]) {
@@ -203,7 +219,7 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     uint32_t x = 0, s = 0;
 
     auto gen = [&](uint64_t i) -> uint32_t {
-        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        const uint64_t r = draw_index(ix, key, i, v, V);
         return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[4]) {
@@ -260,6 +276,142 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     S = s;
 }
 
+// Sorted execution of the packed shape.  The checksums do not depend on the order in which a
+// warp performs its reads, so the warp may take them in an order that is kind to the SM's own
+// translation cache: the stream is cut into epochs of P * R reads, and the reads of an epoch are
+// performed part by part of the window (P equal parts), i.e. the warp walks the epoch's indices
+// P times and each time keeps those that fall into the current part.  At any moment the SM is
+// then working inside 1/P of its window.  Same reads, same words, same checksums; the price is
+// P hashes per read instead of one.  Lines that were kept wait in a small ring in shared memory
+// until 32 of them make a vector for the load loop.
+struct SortedSource {
+    uint32_t *q;
+    uint32_t head, count;          // ring state, warp-uniform
+    uint64_t epoch0, reads;        // first read of the current epoch (relative), reads of the call
+    uint32_t part, batch;          // current part of the window, batch of 32 candidates inside it
+    uint32_t lo, hi;               // index range of the current part
+    bool done;
+    __device__ __forceinline__ void set_part(uint32_t n, uint32_t shift)
+    {
+        lo = (uint32_t)(((uint64_t)n * part) >> shift);
+        hi = (uint32_t)(((uint64_t)n * (part + 1)) >> shift);
+    }
+    __device__ __forceinline__ void init(uint32_t *queue, uint64_t reads_, uint32_t n, uint32_t shift)
+    {
+        q = queue;
+        head = count = 0;
+        epoch0 = 0;
+        reads = reads_;
+        part = batch = 0;
+        done = reads_ == 0;
+        set_part(n, shift);
+    }
+    // Next vector of 32 lines (lane j holds the j-th); entries past the end of the call are junk.
+    __device__ __forceinline__ uint32_t next(const IndexSpec &ix, uint64_t key, uint64_t first,
+                                             uint32_t base, uint32_t n, const Divisor &div,
+                                             uint32_t lane)
+    {
+        const uint32_t parts = 1u << ix.sort_shift;
+        const uint64_t epoch_reads = (uint64_t)ix.sort_reads << ix.sort_shift;
+        while (count < 32u && !done) {
+            const uint64_t t = epoch0 + ((uint64_t)batch << 5) + lane;   // relative read index
+            const uint32_t idx = mod_exact(sm64(key + (first + t) * kGamma), div);
+            const bool keep = t < reads && idx >= lo && idx < hi;
+            const uint32_t m = __ballot_sync(0xFFFFFFFFu, keep);
+            if (keep) q[(head + count + __popc(m & ((1u << lane) - 1u))) & (kSortQueue - 1)] = base + idx;
+            count += __popc(m);
+            // advance: next batch of this part, else next part, else next epoch
+            ++batch;
+            const uint64_t left = reads - epoch0;                       // reads from this epoch on
+            const uint64_t in_epoch = left < epoch_reads ? left : epoch_reads;
+            if (((uint64_t)batch << 5) >= in_epoch) {
+                batch = 0;
+                if (++part == parts) {
+                    part = 0;
+                    epoch0 += in_epoch;
+                    done = epoch0 >= reads;
+                }
+                set_part(n, ix.sort_shift);
+            }
+        }
+        __syncwarp();
+        const uint32_t v = q[(head + lane) & (kSortQueue - 1)];
+        const uint32_t take = count < 32u ? count : 32u;
+        head = (head + take) & (kSortQueue - 1);
+        count -= take;
+        __syncwarp();
+        return v;
+    }
+};
+
+template <int W, int U>
+__device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, uint64_t key,
+                                                  IndexSpec ix, uint64_t first, uint64_t reads,
+                                                  uint32_t base, uint32_t n, uint32_t lane,
+                                                  uint32_t &X, uint32_t &S, BulkRing &br)
+{
+    constexpr int P = 4 / W;     // lines per warp load
+    constexpr int NL = 32 / P;   // warp loads per vector of 32 lines = lanes per line
+    static_assert(W == 1 || W == 2, "16-byte lanes already cover a 512-byte line");
+    static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a vector");
+    const Divisor div = make_divisor(n);
+    SortedSource src;
+    src.init(br.queue, reads, n, ix.sort_shift);
+    const uint32_t sub = lane / NL;
+    const char *lane_ptr = buf + (lane % NL) * 16u;
+    uint32_t d[U][4];
+    uint32_t x = 0, s = 0;
+    auto issue = [&](uint32_t line, uint32_t(&dst)[4]) {
+        load_lane<4>(lane_ptr + (uint64_t)line * (128u * W), dst);
+    };
+    auto clear = [&](uint32_t(&dst)[4]) { dst[0] = dst[1] = dst[2] = dst[3] = 0; };
+    auto fold = [&](const uint32_t(&v)[4]) {
+        x ^= v[0] ^ v[1];
+        x ^= v[2] ^ v[3];
+        s += v[0] + v[1];
+        s += v[2] + v[3];
+    };
+    const uint64_t n_batches = (reads + 31) >> 5;
+    uint32_t cur = src.next(ix, key, first, base, n, div, lane);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u * P + sub);
+        if ((uint64_t)(u * P + sub) < reads) issue(line, d[u]); else clear(d[u]);
+    }
+    for (uint64_t b = 0; b < n_batches; ++b) {
+        const uint64_t t0 = b << 5;
+        const uint32_t nxt = src.next(ix, key, first, base, n, div, lane);
+        if (t0 + 32 + U * P <= reads) {
+#pragma unroll
+            for (int k = 0; k < NL; ++k) {
+                fold(d[k % U]);
+                uint32_t line = (k + U < NL)
+                                    ? __shfl_sync(0xFFFFFFFFu, cur, ((k + U) * P + sub) & 31)
+                                    : __shfl_sync(0xFFFFFFFFu, nxt, ((k + U - NL) * P + sub) & 31);
+                issue(line, d[k % U]);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < NL; ++k) {
+                fold(d[k % U]);
+                uint32_t line = (k + U < NL)
+                                    ? __shfl_sync(0xFFFFFFFFu, cur, ((k + U) * P + sub) & 31)
+                                    : __shfl_sync(0xFFFFFFFFu, nxt, ((k + U - NL) * P + sub) & 31);
+                if (t0 + (uint64_t)((k + U) * P) + sub < reads) issue(line, d[k % U]);
+                else clear(d[k % U]);
+            }
+        }
+        cur = nxt;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        x ^= __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    }
+    X = x;
+    S = s;
+}
+
 // Bulk-copy shape: lane 0 asks the copy engine for each whole line (cp.async.bulk into the warp's
 // ring in shared memory, completion counted on an mbarrier), the lanes then fold the line from
 // shared memory.  One request per line instead of 32 lane requests; same lines, same words.
@@ -281,7 +433,7 @@ __device__ __forceinline__ void warp_reads_bulk(const char *__restrict__ buf, ui
     bool dead = false;      // a wait ran out (warp-uniform)
 
     auto gen = [&](uint64_t i) -> uint32_t {
-        uint64_t r = (ix.mode == RR_INDEX_STRIDE) ? (i * V + v) : sm64(key + i * kGamma);
+        const uint64_t r = draw_index(ix, key, i, v, V);
         return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, int slot) {
@@ -361,6 +513,8 @@ __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_
 {
     if constexpr (VAR == kVarPacked && W < 4)
         warp_reads_packed<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S);
+    else if constexpr (VAR == kVarSorted && W < 4)
+        warp_reads_sorted<W, U>(buf, key, ix, first, reads, base, n, lane, X, S, br);
     else if constexpr (VAR == kVarBulk)
         warp_reads_bulk<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S, br);
     else
@@ -375,7 +529,11 @@ template <int W, int U, int VAR>
 __device__ __forceinline__ BulkRing make_bulk_ring(uint32_t warp, uint32_t lane, uint32_t wpc,
                                                    uint32_t *status)
 {
-    BulkRing br{0u, 0u, 0u, status};
+    BulkRing br{0u, 0u, 0u, status, nullptr};
+    if constexpr (VAR == kVarSorted) {
+        __shared__ uint32_t sh_sort_queue[32 * kSortQueue];
+        br.queue = sh_sort_queue + warp * kSortQueue;
+    }
     if constexpr (VAR == kVarBulk) {
         const uint32_t base = smem_addr(rr_dyn_smem);
         br.ring = base + warp * (U * 128u * W);
@@ -554,6 +712,8 @@ struct ProbeArgs {
 };
 
 constexpr int kProbeUnroll = 8;
+constexpr uint32_t kProbeRendezvousPolls = 1u << 16;  // both limits bound the wait at the start
+constexpr uint64_t kProbeRendezvousNs = 200000;       // 0.2 ms
 
 __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ ProbeArgs a)
 {
@@ -569,13 +729,27 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     if (which >= 2u || sh_slot != 0u) return;  // not on a chosen SM, or not the first block there
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t sm = which ? a.sm_b : a.sm_a;
+    // The two SMs should read side by side for the whole measurement, so the first to arrive
+    // waits for the other.  The wait is bounded: if the other SM gets its block late or never,
+    // this one starts anyway and the host sees a low overlap (or an uncovered SM).
+    if (threadIdx.x == 0 && a.sm_b != 0xFFFFFFFFu) {
+        atomicAdd(&a.rec->ready, 1u);
+        const uint64_t t_wait = globaltimer();
+        bool both = false;
+        for (uint32_t k = 0; k < kProbeRendezvousPolls && !both; ++k) {
+            both = *reinterpret_cast<volatile uint32_t *>(&a.rec->ready) >= 2u;
+            if (!both && globaltimer() - t_wait > kProbeRendezvousNs) break;
+        }
+        if (!both) atomicAdd(&a.rec->gave_up, 1u);
+    }
+    __syncthreads();
     uint64_t t_start = 0;
     if (threadIdx.x == 0) t_start = globaltimer();
     const uint64_t v = (uint64_t)sm * a.wps + warp;
     uint32_t X, S;
-    BulkRing no_ring{0u, 0u, 0u, nullptr};
+    BulkRing no_ring{0u, 0u, 0u, nullptr, nullptr};
     warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
-                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u}, v,
+                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u, 0u, 0u}, v,
                                        (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
                                        a.n_lines, lane, X, S, nullptr, no_ring);
     if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
@@ -602,6 +776,18 @@ static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
         RR_PACKED_ROW(1)
         RR_PACKED_ROW(2)
 #undef RR_PACKED_ROW
+    }
+    if (variant == RR_VARIANT_SORTED && W < 4) {
+        if (W == 1) switch (U) {
+                case 1: return read_kernel<1, 1, kVarSorted>;
+                case 4: return read_kernel<1, 4, kVarSorted>;
+                default: return read_kernel<1, 2, kVarSorted>;
+            }
+        switch (U) {
+            case 1: return read_kernel<2, 1, kVarSorted>;
+            case 4: return read_kernel<2, 4, kVarSorted>;
+            default: return read_kernel<2, 2, kVarSorted>;
+        }
     }
     if (variant == RR_VARIANT_L2_128 || variant == RR_VARIANT_L2_256 ||
         variant == RR_VARIANT_BULK) {  // comparison variants: ring depth 4 or 8 only
@@ -655,9 +841,21 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
 {
     if (!p || !out || !scratch || !p->buf) return RR_ERR_ARG;
     if (!width_ok(p->words_per_lane) || p->mode > RR_MODE_POOLED ||
-        p->index_mode > RR_INDEX_PHASED || p->variant > RR_VARIANT_BULK)
+        p->index_mode > RR_INDEX_MIXED || p->variant > RR_VARIANT_SORTED)
         return RR_ERR_ARG;
-    if (p->reserved) return RR_ERR_ARG;
+    if (p->variant == RR_VARIANT_SORTED) {
+        const uint32_t P = p->sort_parts, R = p->sort_reads;
+        if (p->words_per_lane == 4 || p->index_mode != RR_INDEX_RANDOM) return RR_ERR_ARG;
+        if (P < 2 || P > 64 || (P & (P - 1)) || R < 32 || R % 32u || R > (1u << 20)) return RR_ERR_ARG;
+    } else if (p->sort_parts || p->sort_reads) {
+        return RR_ERR_ARG;
+    }
+    if (p->index_mode == RR_INDEX_MIXED) {
+        const uint32_t k = p->mix_period;
+        if (k == 0 || (k & (k - 1)) || k > (1u << 20)) return RR_ERR_ARG;
+    } else if (p->mix_period) {
+        return RR_ERR_ARG;
+    }
     if (p->index_mode == RR_INDEX_PHASED) {
         const uint32_t b = p->phase_reads;
         if (b < 32 || (b & (b - 1)) || p->first_read % 32u) return RR_ERR_ARG;
@@ -666,9 +864,10 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
         return RR_ERR_ARG;
     }
     if (p->mode != RR_MODE_POOLED && (p->pool_block_reads || p->warp_start)) return RR_ERR_ARG;
-    uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_PACKED ? 4u : 8u);
-    if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && p->variant == RR_VARIANT_PACKED))
-        return RR_ERR_ARG;
+    const bool packed_shape = p->variant == RR_VARIANT_PACKED || p->variant == RR_VARIANT_SORTED;
+    uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_SORTED ? 2u : packed_shape ? 4u : 8u);
+    if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && packed_shape)) return RR_ERR_ARG;
+    if (p->variant == RR_VARIANT_SORTED && U > 4) return RR_ERR_ARG;
     if ((p->variant == RR_VARIANT_L2_128 || p->variant == RR_VARIANT_L2_256) && U != 8)
         return RR_ERR_ARG;
     if (p->variant == RR_VARIANT_BULK && U != 4 && U != 8) return RR_ERR_ARG;
@@ -782,11 +981,8 @@ static int32_t search_ballast(const void *kernel, int block, int want, size_t ne
     RR_CUDA(cudaFuncGetAttributes(&fa, kernel));
     const int per_block_reserved = 1024;
     const int stat = (int)fa.sharedSizeBytes;
-    int lo = f.smem_per_sm / (want + 1) - per_block_reserved - stat + 1;
-    if (lo < 0) lo = 0;
-    const int hi = std::min(f.smem_per_block_optin - stat,
-                            f.smem_per_sm / want - per_block_reserved - stat);
-    if ((int)need > hi) {
+    const int most = f.smem_per_block_optin - stat;  // the largest request one block may make
+    if ((int)need > most) {
         set_cuda_error(cudaErrorLaunchOutOfResources, "shared-memory ring does not fit");
         return RR_ERR_CUDA;
     }
@@ -794,16 +990,19 @@ static int32_t search_ballast(const void *kernel, int block, int want, size_t ne
     // is a permission, it does not change residency
     g_n_attribute_sets.fetch_add(1);
     RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 std::max(hi, 0)));
+                                 std::max(most, 0)));
+    if (want <= 0) {  // no residency requirement (LOGICAL mode): just the ring
+        *smem_out = need;
+        return RR_OK;
+    }
     auto blocks_at = [&](size_t smem, int *nb) -> int32_t {
         g_n_occupancy_queries.fetch_add(1);
         RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, kernel, block, smem));
         return RR_OK;
     };
-    if (want <= 0) {  // no residency requirement (LOGICAL mode): just the ring
-        *smem_out = need;
-        return RR_OK;
-    }
+    int lo = f.smem_per_sm / (want + 1) - per_block_reserved - stat + 1;
+    if (lo < 0) lo = 0;
+    const int hi = std::min(most, f.smem_per_sm / want - per_block_reserved - stat);
     for (int smem = std::max(lo, (int)need); smem <= hi; smem += 1024) {
         int nb = 0;
         int32_t rc = blocks_at((size_t)smem, &nb);
@@ -883,6 +1082,11 @@ static void make_launch_args(const rr_read_params_t *p, const Geometry &g, const
     a->ix.sub_lines = 0;
     a->ix.sm = 0;
     a->ix.nsm = 0;  // set by the block in per-SM mode
+    a->ix.sort_shift = 0;
+    a->ix.sort_reads = p->sort_reads;
+    while ((1u << a->ix.sort_shift) < p->sort_parts) ++a->ix.sort_shift;
+    if (p->index_mode == RR_INDEX_MIXED)
+        while ((1u << a->ix.phase_shift) < p->mix_period) ++a->ix.phase_shift;
     if (p->index_mode == RR_INDEX_PHASED) {
         while ((1u << a->ix.phase_shift) < p->phase_reads) ++a->ix.phase_shift;
         const uint64_t sub = p->phase_window_bytes / (128ull * p->words_per_lane);
@@ -1091,22 +1295,80 @@ static ProbeArgs probe_args(const void *buf, uint64_t region_bytes, uint32_t a, 
 static bool probe_rate(const ProbeRecord &r, bool solo, uint64_t total_reads, double *gbps,
                        double *seconds, double *overlap)
 {
+    return rr_probe_rate(r.t_start, r.t_end, r.claim, solo ? 1u : 0u, total_reads, gbps, seconds,
+                         overlap) == RR_OK;
+}
+
+}  // namespace rr
+
+// Bytes of both SMs over the union of their intervals; overlap = intersection / union.
+extern "C" int32_t rr_probe_rate(const uint64_t *t_start, const uint64_t *t_end,
+                                 const uint32_t *claim, uint32_t solo, uint64_t total_reads,
+                                 double *gbps, double *seconds, double *overlap)
+{
+    if (!t_start || !t_end || !claim || !gbps || !seconds || !overlap || solo > 1) return RR_ERR_ARG;
     const int k = solo ? 1 : 2;
-    uint64_t s_min = ~0ull, s_max = 0, e_min = ~0ull, e_max = 0;
+    uint64_t first_start = ~0ull, last_start = 0, first_end = ~0ull, last_end = 0;
     for (int i = 0; i < k; ++i) {
-        if (r.claim[i] == 0 || r.t_end[i] == 0) return false;
-        s_min = std::min(s_min, r.t_start[i]);
-        s_max = std::max(s_max, r.t_start[i]);
-        e_min = std::min(e_min, r.t_end[i]);
-        e_max = std::max(e_max, r.t_end[i]);
+        if (claim[i] == 0 || t_end[i] == 0 || t_end[i] < t_start[i]) return RR_ERR_SM_UNCOVERED;
+        first_start = std::min(first_start, t_start[i]);
+        last_start = std::max(last_start, t_start[i]);
+        first_end = std::min(first_end, t_end[i]);
+        last_end = std::max(last_end, t_end[i]);
     }
-    const double span = (double)(e_max - s_min) * 1e-9;
-    const uint64_t bytes = (total_reads / 2) * k * 128ull;
-    *seconds = span;
-    *gbps = span > 0 ? (double)bytes / span * 1e-9 : 0.0;
-    *overlap = (e_max > s_min && e_min > s_max) ? (double)(e_min - s_max) / (double)(e_max - s_min)
-                                                : 0.0;
-    return true;
+    const uint64_t uni = last_end - first_start;
+    const uint64_t bytes = (total_reads / 2) * (uint64_t)k * 128ull;
+    *seconds = (double)uni * 1e-9;
+    *gbps = uni ? (double)bytes / (double)uni : 0.0;  // bytes per ns = GB/s
+    *overlap = (uni && first_end > last_start) ? (double)(first_end - last_start) / (double)uni : 0.0;
+    return RR_OK;
+}
+
+namespace rr {
+
+// A pair whose two SMs did not run side by side for at least this share of the measurement is
+// measured again with more reads.
+constexpr double kProbeOverlapGoal = 0.98;
+constexpr int kProbeMaxDoublings = 3;
+
+}  // namespace rr
+
+namespace rr {
+
+struct ProbeSample {
+    double gbps, seconds, overlap, seconds_event;
+};
+
+// One probe launch on its own (synchronous), retried with larger grids if a chosen SM got no
+// block.  `rec` is the record on the device the launch writes.
+static int32_t probe_once(const void *buf, uint64_t region_bytes, uint32_t sm_a, uint32_t sm_b,
+                          uint64_t total_reads, uint32_t wps, uint64_t seed, void *out_dev,
+                          ProbeRecord *rec, const DeviceFacts &f, size_t smem, cudaStream_t stream,
+                          ProbeSample *out)
+{
+    EventPair *ev = nullptr;
+    int32_t rc = timing_events(f.device, &ev);
+    if (rc != RR_OK) return rc;
+    const ProbeArgs pa = probe_args(buf, region_bytes, sm_a, sm_b, total_reads, wps, seed, out_dev,
+                                    rec, f.nsm);
+    for (int attempt = 0; attempt < 3; ++attempt) {
+        RR_CUDA(cudaMemsetAsync(rec, 0, sizeof(ProbeRecord), stream));
+        RR_CUDA(cudaMemsetAsync(out_dev, 0, 2ull * wps * sizeof(uint2), stream));
+        RR_CUDA(cudaEventRecord(ev->e0, stream));
+        probe_kernel<<<(uint32_t)f.nsm * (4u << attempt), wps * 32, smem, stream>>>(pa);
+        RR_CUDA(cudaGetLastError());
+        RR_CUDA(cudaEventRecord(ev->e1, stream));
+        ProbeRecord h;
+        RR_CUDA(cudaMemcpyAsync(&h, rec, sizeof(h), cudaMemcpyDeviceToHost, stream));
+        RR_CUDA(cudaStreamSynchronize(stream));
+        float ms = 0.f;
+        RR_CUDA(cudaEventElapsedTime(&ms, ev->e0, ev->e1));
+        if (probe_rate(h, sm_a == sm_b, total_reads, &out->gbps, &out->seconds, &out->overlap)) {
+            out->seconds_event = (double)ms * 1e-3;
+            return RR_OK;
+        }
+    }
+    return RR_ERR_SM_UNCOVERED;
 }
 
 }  // namespace rr
@@ -1122,51 +1384,21 @@ extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_
     rc = device_facts(&f);
     if (rc != RR_OK) return rc;
     if (sm_a >= (uint32_t)f.nsm || sm_b >= (uint32_t)f.nsm) return RR_ERR_ARG;
-    cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
     rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
     if (rc != RR_OK) return rc;
-    ProbeRecord *rec = &((ScratchHeader *)scratch_dev)->probe;
-    ProbeArgs pa = probe_args(buf, region_bytes, sm_a, sm_b, total_reads, wps, seed, out_dev, rec,
-                              f.nsm);
-    EventPair *ev = nullptr;
-    rc = timing_events(f.device, &ev);
-    if (rc != RR_OK) return rc;
-    cudaEvent_t e0 = ev->e0, e1 = ev->e1;
-    int32_t result = RR_ERR_SM_UNCOVERED;
     std::memset(res, 0, sizeof(*res));
-    for (int attempt = 0; attempt < 3 && result == RR_ERR_SM_UNCOVERED; ++attempt) {
-        cudaError_t e = cudaMemsetAsync(rec, 0, sizeof(ProbeRecord), stream);
-        if (e == cudaSuccess) e = cudaMemsetAsync(out_dev, 0, 2ull * wps * sizeof(uint2), stream);
-        if (e == cudaSuccess) e = cudaEventRecord(e0, stream);
-        if (e == cudaSuccess) {
-            probe_kernel<<<(uint32_t)f.nsm * (4u << attempt), wps * 32, smem, stream>>>(pa);
-            e = cudaGetLastError();
-        }
-        if (e == cudaSuccess) e = cudaEventRecord(e1, stream);
-        ProbeRecord h;
-        if (e == cudaSuccess)
-            e = cudaMemcpyAsync(&h, rec, sizeof(h), cudaMemcpyDeviceToHost, stream);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-        float ms = 0.f;
-        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
-        if (e != cudaSuccess) {
-            set_cuda_error(e, "rr_probe_pair");
-            result = RR_ERR_CUDA;
-            break;
-        }
-        double gbps, sec, ov;
-        if (probe_rate(h, sm_a == sm_b, total_reads, &gbps, &sec, &ov)) {
-            res->seconds_event = (double)ms * 1e-3;
-            res->seconds_device = sec;
-            res->bytes = (total_reads / 2) * (sm_a == sm_b ? 1 : 2) * 128ull;
-            res->gbps = gbps;
-            res->sms_covered = sm_a == sm_b ? 1 : 2;
-            res->blocks_run = res->sms_covered;
-            result = RR_OK;
-        }
-    }
-    return result;
+    ProbeSample s;
+    rc = probe_once(buf, region_bytes, sm_a, sm_b, total_reads, wps, seed, out_dev,
+                    &((ScratchHeader *)scratch_dev)->probe, f, smem, (cudaStream_t)stream_, &s);
+    if (rc != RR_OK) return rc;
+    res->seconds_event = s.seconds_event;
+    res->seconds_device = s.seconds;
+    res->bytes = (total_reads / 2) * (sm_a == sm_b ? 1 : 2) * 128ull;
+    res->gbps = s.gbps;
+    res->sms_covered = sm_a == sm_b ? 1 : 2;
+    res->blocks_run = res->sms_covered;
+    return RR_OK;
 }
 
 extern "C" size_t rr_probe_matrix_scratch_bytes(uint32_t nsm)
@@ -1174,14 +1406,17 @@ extern "C" size_t rr_probe_matrix_scratch_bytes(uint32_t nsm)
     return sizeof(ScratchHeader) + sizeof(ProbeRecord) * ((size_t)nsm * (nsm + 1) / 2);
 }
 
-extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint64_t total_reads,
-                                   uint32_t wps, uint64_t seed, uint32_t repeats, float *T_host,
-                                   uint32_t nsm, void *out_dev, void *scratch_dev,
-                                   double *overlap_min_host, void *stream_)
+extern "C" int32_t rr_probe_rows(const void *buf, uint64_t region_bytes, uint64_t total_reads,
+                                 uint32_t wps, uint64_t seed, uint32_t repeats, uint32_t row_begin,
+                                 uint32_t row_end, float *T_host, uint32_t nsm, void *out_dev,
+                                 void *scratch_dev, rr_probe_stats_t *stats, float *overlap_host,
+                                 void *stream_)
 {
     int32_t rc = validate_probe(buf, region_bytes, total_reads, wps, out_dev, scratch_dev);
     if (rc != RR_OK) return rc;
     if (!T_host || repeats == 0 || repeats > 64 || nsm < 2 || nsm > RR_MAX_SM) return RR_ERR_ARG;
+    if (row_begin >= row_end || row_end > nsm) return RR_ERR_ARG;
+    if (total_reads > (1ull << 58)) return RR_ERR_RANGE;  // room for the doublings
     DeviceFacts f;
     rc = device_facts(&f);
     if (rc != RR_OK) return rc;
@@ -1191,24 +1426,29 @@ extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint6
     rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
     if (rc != RR_OK) return rc;
 
-    const size_t n_pairs = (size_t)nsm * (nsm + 1) / 2;
+    size_t n_pairs = 0;  // pairs (a, b >= a) of the requested rows
+    for (uint32_t a = row_begin; a < row_end; ++a) n_pairs += nsm - a;
     ProbeRecord *recs = (ProbeRecord *)((char *)scratch_dev + sizeof(ScratchHeader));
+    ProbeRecord *solo_rec = &((ScratchHeader *)scratch_dev)->probe;
     std::vector<ProbeRecord> h(n_pairs);
     std::vector<float> samples(n_pairs * repeats);
-    double overlap_min = 1.0;
+    std::vector<float> worst(n_pairs, 1.0f);  // smallest kept overlap of each pair over the repeats
+    rr_probe_stats_t st;
+    std::memset(&st, 0, sizeof(st));
+    st.overlap_min = 1.0;
     // untimed warm-up: the first launches after idle (cold translation caches, clock ramp) run
     // slow and would plant outliers in the first row
     for (int w = 0; w < 16; ++w) {
         ProbeArgs pa = probe_args(buf, region_bytes, (uint32_t)w % nsm, nsm - 1 - (uint32_t)w % nsm,
-                                  total_reads, wps, seed, out_dev,
-                                  &((ScratchHeader *)scratch_dev)->probe, f.nsm);
+                                  total_reads, wps, seed, out_dev, solo_rec, f.nsm);
+        RR_CUDA(cudaMemsetAsync(solo_rec, 0, sizeof(ProbeRecord), stream));
         probe_kernel<<<nsm * 4u, wps * 32, smem, stream>>>(pa);
     }
     RR_CUDA(cudaGetLastError());
     for (uint32_t rep = 0; rep < repeats; ++rep) {
         RR_CUDA(cudaMemsetAsync(recs, 0, sizeof(ProbeRecord) * n_pairs, stream));
         size_t k = 0;
-        for (uint32_t a = 0; a < nsm; ++a)
+        for (uint32_t a = row_begin; a < row_end; ++a)
             for (uint32_t b = a; b < nsm; ++b, ++k) {
                 ProbeArgs pa = probe_args(buf, region_bytes, a, b, total_reads, wps, seed, out_dev,
                                           recs + k, f.nsm);
@@ -1219,33 +1459,63 @@ extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint6
                                 cudaMemcpyDeviceToHost, stream));
         RR_CUDA(cudaStreamSynchronize(stream));
         k = 0;
-        for (uint32_t a = 0; a < nsm; ++a)
+        for (uint32_t a = row_begin; a < row_end; ++a)
             for (uint32_t b = a; b < nsm; ++b, ++k) {
-                double gbps, sec, ov;
-                if (!probe_rate(h[k], a == b, total_reads, &gbps, &sec, &ov)) {
+                ProbeSample best{0, 0, 0, 0};
+                bool have = probe_rate(h[k], a == b, total_reads, &best.gbps, &best.seconds,
+                                       &best.overlap);
+                if (!have) {
                     // a chosen SM got no block in the queued launch: redo this pair on its own
-                    rr_result_t r;
-                    rc = rr_probe_pair(buf, region_bytes, a, b, total_reads, wps, seed, out_dev,
-                                       scratch_dev, &r, stream_);
+                    rc = probe_once(buf, region_bytes, a, b, total_reads, wps, seed, out_dev,
+                                    solo_rec, f, smem, stream, &best);
                     if (rc != RR_OK) return rc;
-                    gbps = r.gbps;
-                    ov = 1.0;
+                    ++st.relaunched;
                 }
-                if (a != b) overlap_min = std::min(overlap_min, ov);
-                samples[k * repeats + rep] = (float)gbps;
+                if (a != b) {
+                    // the two SMs must read side by side: while they did not, measure again with
+                    // twice the reads -- at most three times, and only while doubling still helps
+                    double prev = best.overlap;
+                    for (int d = 1; d <= kProbeMaxDoublings && best.overlap < kProbeOverlapGoal; ++d) {
+                        ProbeSample s;
+                        rc = probe_once(buf, region_bytes, a, b, total_reads << d, wps, seed,
+                                        out_dev, solo_rec, f, smem, stream, &s);
+                        if (rc != RR_OK) return rc;
+                        ++st.reruns;
+                        if (s.overlap > best.overlap) best = s;
+                        if (s.overlap < prev + 0.01) break;  // not start skew: the SMs differ in speed
+                        prev = s.overlap;
+                    }
+                    worst[k] = std::min(worst[k], (float)best.overlap);
+                    st.overlap_min = std::min(st.overlap_min, best.overlap);
+                }
+                samples[k * repeats + rep] = (float)best.gbps;
             }
     }
     size_t k = 0;
-    for (uint32_t a = 0; a < nsm; ++a)
+    for (uint32_t a = row_begin; a < row_end; ++a)
         for (uint32_t b = a; b < nsm; ++b, ++k) {
             float *s = &samples[k * repeats];
             std::sort(s, s + repeats);
             const float med = s[(repeats - 1) / 2];
             T_host[(size_t)a * nsm + b] = med;
             T_host[(size_t)b * nsm + a] = med;
+            if (a != b && worst[k] < (float)kProbeOverlapGoal) ++st.pairs_below_goal;
+            if (overlap_host) {
+                overlap_host[(size_t)a * nsm + b] = worst[k];
+                overlap_host[(size_t)b * nsm + a] = worst[k];
+            }
         }
-    if (overlap_min_host) *overlap_min_host = overlap_min;
+    if (stats) *stats = st;
     return RR_OK;
+}
+
+extern "C" int32_t rr_probe_matrix(const void *buf, uint64_t region_bytes, uint64_t total_reads,
+                                   uint32_t wps, uint64_t seed, uint32_t repeats, float *T_host,
+                                   uint32_t nsm, void *out_dev, void *scratch_dev,
+                                   rr_probe_stats_t *stats, float *overlap_host, void *stream_)
+{
+    return rr_probe_rows(buf, region_bytes, total_reads, wps, seed, repeats, 0, nsm, T_host, nsm,
+                         out_dev, scratch_dev, stats, overlap_host, stream_);
 }
 
 // ---- rr_random_read_static: the same read with built-in scratch ---------------------------------

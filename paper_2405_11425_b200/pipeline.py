@@ -1,8 +1,9 @@
 """The paper's experiments strung together over the C-ABI entry points.
 
-Nothing here computes on the data path: every read, probe and clustering step is a call into
-librr (see binding.py).  This module only owns device buffers (torch), picks sizes, and keeps
-the bookkeeping of a run:
+Nothing here computes on the data path or decides a plan: every read, probe and clustering step,
+and every rule that turns measurements into windows, weights or sizes, is a call into librr (see
+binding.py).  This module only owns device buffers (torch), loops over sizes, and keeps the
+bookkeeping of a run:
 
   Session.fill()            Section 2.1 needs a region with known contents       (rr_fill)
   Session.read()            one random-read launch, grouped or not               (rr_random_read)
@@ -32,6 +33,7 @@ class Groups:
     overlap_min: float = 1.0
     probe_seconds: float = 0.0
     sizes: list = field(default_factory=list)
+    probe_stats: dict = field(default_factory=dict)
 
 
 @dataclass
@@ -92,27 +94,6 @@ def load_calibration(path, uuid: str, nsm: int):
     return groups, reach, None if w is None else np.asarray(w, dtype=np.uint32)
 
 
-def rebalanced_weights(work, finish_ns, scale: int = 1_000_000) -> np.ndarray:
-    """New integer group weights from one balanced-run observation: a group that did `work`
-    units and finished after `finish_ns` has shown a rate work/finish; weights are those rates,
-    normalised to sum to about `scale`.  Groups that were not seen (finish 0) keep a token weight
-    of one thousandth of the slowest observed rate."""
-    work = np.asarray(work, dtype=np.float64)
-    finish = np.asarray(finish_ns, dtype=np.float64)
-    rate = np.where(finish > 0, work / np.maximum(finish, 1.0), 0.0)
-    if not (rate > 0).any():
-        raise ValueError("no group finished any work")
-    rate = np.maximum(rate, rate[rate > 0].min() * 1e-3)
-    return np.maximum(1, np.rint(rate / rate.sum() * scale)).astype(np.uint32)
-
-
-def finish_spread(finish_ns) -> float:
-    """(latest - earliest) / latest over the groups that ran."""
-    f = np.asarray(finish_ns, dtype=np.float64)
-    f = f[f > 0]
-    return float((f.max() - f.min()) / f.max()) if f.size else 0.0
-
-
 class Session:
     """Device buffers of one GPU plus the calls of the path."""
 
@@ -120,13 +101,13 @@ class Session:
                  max_warps_per_sm: int = 32):
         import torch
         self.torch = torch
-        self.info = rr.rr_device_info()
+        # small buffers first, so the region can take what is left
+        self.scratch = torch.zeros(rr.rr_scratch_bytes(), dtype=torch.uint8, device="cuda")
+        self.info = rr.rr_device_info(self.scratch)
         self.nsm = int(self.info["nsm_prop"])
         if self.info["nsm_reg"] != self.nsm:
             raise RuntimeError(f"%nsmid = {self.info['nsm_reg']} but the device reports "
                                f"{self.nsm} SMs")
-        # small buffers first, so the region can take what is left
-        self.scratch = torch.zeros(rr.rr_scratch_bytes(), dtype=torch.uint8, device="cuda")
         self.probe_scratch = torch.zeros(rr.rr_probe_matrix_scratch_bytes(self.nsm),
                                          dtype=torch.uint8, device="cuda")
         self.out = torch.zeros((self.nsm * max_warps_per_sm, 2), dtype=torch.int32, device="cuda")
@@ -222,68 +203,99 @@ class Session:
         return pts
 
     def measure_reach(self, sizes_gib=(1, 4, 16, 32, 48, 64, 96, 128, 160), *, seed: int = 7,
-                      refine_gib: int = 2, **kw) -> Reach:
-        """Size sweep, then bisection at `refine_gib` granularity between the last size at or
-        above 0.9 plateau and the first below it."""
+                      refine_gib: int = 2, sustained: bool = True, **kw) -> Reach:
+        """Size sweep, then refinement at `refine_gib` granularity: rr_reach_next names the next
+        size to measure until it has none left.  With `sustained` every point is measured by the
+        settle-then-time protocol (>= 50 ms of kernel time, 5 regions), else by short bursts."""
         sizes = [s * GiB for s in sizes_gib if s * GiB < self.region_bytes] + [self.region_bytes]
-        pts = self.size_sweep(sizes, seed=seed, **kw)
-        cliff, plateau, reach = rr.rr_reach([p[0] for p in pts], [p[1] for p in pts])
-        if cliff:
-            good = reach
-            bad = min(p[0] for p in pts if p[0] > reach)
-            step = refine_gib * GiB
-            while bad - good > step:
-                mid = ((good + bad) // 2 // step) * step
-                if mid <= good or mid >= bad:
-                    break
-                g, _ = self.read(mid, seed=seed, reads_per_warp=256 * 16, **kw)
-                pts.append((mid, g))
-                if g >= 0.9 * plateau:
-                    good = mid
-                else:
-                    bad = mid
-            pts.sort()
-            cliff, plateau, reach = rr.rr_reach([p[0] for p in pts], [p[1] for p in pts])
-        return Reach(cliff, plateau, reach, pts)
+
+        def rate(n):
+            if not sustained:
+                return self.read(n, seed=seed, reads_per_warp=256 * 16, **kw)[0]
+            p = self.params(n, seed=seed, reads_per_warp=256 * 16, **kw)
+            return self.sustained(p, settle=20, min_ms=50.0, reps=5)["gbps"]
+
+        pts = {int(n): rate(n) for n in sizes}
+        for _ in range(64):
+            xs = sorted(pts)
+            nxt = rr.rr_reach_next(xs, [pts[x] for x in xs], refine_gib * GiB)
+            if not nxt or nxt in pts:
+                break
+            pts[nxt] = rate(nxt)
+        xs = sorted(pts)
+        cliff, plateau, reach = rr.rr_reach(xs, [pts[x] for x in xs])
+        return Reach(cliff, plateau, reach, [(x, pts[x]) for x in xs])
 
     def measure_sm_reach(self, sizes_mib=(32, 64, 128, 256, 384, 512, 768, 1024), *,
                          keep: float = 0.97, seed: int = 23, reads_per_warp: int = 256 * 16):
         """How large a window can one SM read at random before its own translation cache stops
         covering it?  Every SM gets a window of the given size (windows spread over the buffer,
-        equal work); the answer is the largest size whose rate stays within `keep` of the rate
-        at the smallest sizes.  Returns (reach_bytes, [(size_bytes, GB/s)])."""
+        equal work); rr_sm_reach turns the rates into the answer.
+        Returns (reach_bytes, [(size_bytes, GB/s)])."""
         ids = np.arange(self.nsm, dtype=np.uint16)
         stride = (self.region_bytes // 128) // self.nsm
         pts = []
         for mib in sizes_mib:
             n = min((mib << 20) // 128, stride)
+            if pts and int(n) * 128 <= pts[-1][0]:
+                continue
             win = np.array([[k * stride, n] for k in range(self.nsm)], np.uint32)
             g, _ = self.read(self.region_bytes, seed=seed, reads_per_warp=reads_per_warp,
                              group_of_sm=ids, windows=win)
             pts.append((int(n) * 128, g))
-        top = sorted(p[1] for p in pts[:3])[1]
-        reach = pts[0][0]
-        for size, g in pts:
-            if g >= keep * top:
-                reach = size
-            else:
-                break
+        reach = rr.rr_sm_reach([p[0] for p in pts], [p[1] for p in pts], keep)
         return reach, pts
 
     # -- groups -----------------------------------------------------------------------------
     def discover_groups(self, *, probe_region_bytes=None, total_reads: int = 1 << 18,
                         warps_per_sm: int = 32, seed: int = 5, repeats: int = 3,
-                        solo_normalise: bool = True) -> Groups:
+                        solo_normalise: bool = True, checkpoint=None,
+                        rows_per_block: int = 16) -> Groups:
+        """Pair-probe matrix, then clustering.  With `checkpoint` (a path) the matrix is probed in
+        blocks of rows and saved after each block; a later call with the same card and probe
+        settings picks up after the last finished block instead of starting over."""
         import time
         region = probe_region_bytes or self.region_bytes
         t0 = time.time()
-        T, overlap = rr.rr_probe_matrix(self.buf, region, total_reads, warps_per_sm, seed, repeats,
-                                        self.nsm, self.probe_out, self.probe_scratch)
+        if checkpoint is None:
+            T, stats = rr.rr_probe_matrix(self.buf, region, total_reads, warps_per_sm, seed,
+                                          repeats, self.nsm, self.probe_out, self.probe_scratch)
+        else:
+            T, stats = self._probe_with_checkpoint(checkpoint, region, total_reads, warps_per_sm,
+                                                   seed, repeats, rows_per_block)
         dt = time.time() - t0
         flags = rr.RR_CLUSTER_SOLO_NORMALISE if solo_normalise else 0
         g, n_groups, conf, _ = rr.rr_cluster(T, self.scratch, flags)
-        return Groups(g.astype(np.uint16), n_groups, conf, T, overlap, dt,
-                      np.bincount(g, minlength=n_groups).tolist())
+        return Groups(g.astype(np.uint16), n_groups, conf, T, stats["overlap_min"], dt,
+                      np.bincount(g, minlength=n_groups).tolist(), stats)
+
+    def _probe_with_checkpoint(self, path, region, total_reads, wps, seed, repeats, rows_per_block):
+        import json
+        from pathlib import Path
+        path = Path(path)
+        meta = {"uuid": self.info["uuid"], "nsm": self.nsm, "region_bytes": int(region),
+                "total_reads": int(total_reads), "warps_per_sm": int(wps), "seed": int(seed),
+                "repeats": int(repeats)}
+        T = np.zeros((self.nsm, self.nsm), dtype=np.float32)
+        done = 0
+        stats = {"overlap_min": 1.0, "pairs_below_goal": 0, "reruns": 0, "relaunched": 0}
+        if path.exists():
+            with np.load(path, allow_pickle=False) as z:
+                if json.loads(str(z["meta"])) == meta:          # same card, same probe settings
+                    T = np.ascontiguousarray(z["T"], dtype=np.float32)
+                    done = int(z["rows_done"])
+                    stats = json.loads(str(z["stats"]))
+        while done < self.nsm:
+            end = min(self.nsm, done + max(1, rows_per_block))
+            st = rr.rr_probe_rows(self.buf, region, total_reads, wps, seed, repeats, done, end, T,
+                                  self.probe_out, self.probe_scratch)
+            stats = {"overlap_min": min(stats["overlap_min"], st["overlap_min"]),
+                     **{k: stats[k] + st[k] for k in ("pairs_below_goal", "reruns", "relaunched")}}
+            done = end
+            tmp = path.with_suffix(".tmp.npz")
+            np.savez(tmp, T=T, rows_done=done, meta=json.dumps(meta), stats=json.dumps(stats))
+            tmp.replace(path)
+        return T, stats
 
     # -- windows-------------------------------------------------------------------------------
     def windows(self, groups: Groups, window_bytes: int, W: int = 1, region_bytes=None):
@@ -303,20 +315,11 @@ class Session:
             rates.append(rate)
         return rates
 
-    def balanced_plan(self, groups: Groups, rates, n_warps: int, *, W: int = 1,
-                      max_window_bytes: int = 0, region_bytes=None):
-        """Windows and logical-warp ranges in proportion to the groups' measured rates
-        (weights = rates in MB/s).  Returns (windows, warp_start)."""
-        weights = np.maximum(1, np.rint(np.asarray(rates, dtype=np.float64) * 1000.0)).astype(
-            np.uint32)
-        return rr.rr_make_weighted_windows(region_bytes or self.region_bytes, W, weights, n_warps,
-                                           max_window_bytes)
-
     def balance(self, groups: Groups, *, W: int = 1, n_warps: int | None = None,
                 reads_per_warp: int = 256 * 64, seed: int = 23, max_window_bytes: int = 0,
                 rounds: int = 6, spread_goal: float = 0.02, start_rates=None,
                 launches_per_round: int = 1, **kw):
-        """Closed-loop version of balanced_plan: run the pooled workload, see from the per-SM
+        """Closed loop: run the pooled workload, see from the per-SM
         timers when each group finished, move work (and window size) towards the groups that
         finished early, repeat.  Needed because a group's capacity with every other group
         running differs from its capacity alone.  Stops after `rounds` rounds or once the
@@ -342,17 +345,12 @@ class Session:
             for _ in range(max(1, launches_per_round)):
                 rr.rr_random_read(p, self.out, self.scratch, timed=False)
             t0, t1 = rr.rr_read_block_times(self.scratch, self.nsm)
-            ran = t1 > 0
-            begin = t0[ran].min()
-            history.append(n_warps * reads_per_warp * 128 * W / float(t1[ran].max() - begin))
-            work = np.diff(ws.astype(np.int64)).astype(np.float64)
-            finish = np.zeros(G)
-            for g in range(G):
-                m = (groups.group_of_sm == g) & ran
-                finish[g] = max(1.0, float(t1[m].max() - begin)) if m.any() else 0.0
-            if finish_spread(finish) <= spread_goal:
+            finish, span_ns = rr.rr_group_finish(t0, t1, groups.group_of_sm, G)
+            history.append(n_warps * reads_per_warp * 128 * W / max(span_ns, 1))
+            work = np.diff(ws.astype(np.int64)).astype(np.uint32)
+            if rr.rr_finish_spread_ppm(finish) <= int(spread_goal * 1e6):
                 break
-            weights = rebalanced_weights(work, finish)
+            weights = rr.rr_rebalance_weights(work, finish)
         win, ws = rr.rr_make_weighted_windows(self.region_bytes, W, weights, n_warps,
                                               max_window_bytes)
         return win, ws, weights, history
@@ -380,11 +378,8 @@ class Session:
         A window per SM is still a window per group in the paper's sense (every group's
         footprint stays below its reach), and it lets each SM's own small translation cache
         catch a share of the lookups before they reach the group's shared path."""
-        order = np.argsort(groups.group_of_sm, kind="stable")
-        ids = np.empty(self.nsm, dtype=np.uint16)
-        ids[order] = np.arange(self.nsm, dtype=np.uint16)
-        return Groups(ids, self.nsm, groups.confidence, None, groups.overlap_min, 0.0,
-                      [1] * self.nsm)
+        ids, n = rr.rr_owner_map(groups.group_of_sm)
+        return Groups(ids, n, groups.confidence, None, groups.overlap_min, 0.0, [1] * n)
 
     def naive_control(self, window_bytes: int, seed: int, W: int = 1, region_bytes=None):
         """The paper's per-SM control: every SM on its own picks a pseudo-random chunk."""

@@ -8,7 +8,8 @@ Experiments (paper section -> BASELINE config):
   pair probe + clustering             Section 2.2, Fig. 2-3          configs[3]
   single groups, group pairs          Section 2.3, Fig. 4-5
   grouped windows over all memory     Section 2.4, Fig. 6            configs[4]
-  sequential reads of the same kernel Section 2.1 ("even better")
+  sequential reads of the same kernel Section 2.1 (last paragraph)
+  allocation paths (--alloc-study)    Section 1.2 (reach = translations x page size)
 All numbers are event-timed GB/s (10^9 B/s), median of the repetitions; nothing is computed here
 beyond bookkeeping.
 """
@@ -32,7 +33,7 @@ def _stats(ses, region, reps=5, **kw):
     return {"median": r[(len(r) - 1) // 2], "min": r[0], "max": r[-1]}
 
 
-def run(out_dir: Path, quick: bool = False) -> dict:
+def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     import torch
     torch.cuda.set_device(0)
     out_dir.mkdir(parents=True, exist_ok=True)
@@ -145,6 +146,13 @@ def run(out_dir: Path, quick: bool = False) -> dict:
             rows[name]["naive_per_sm_control"] = _stats(ses, N, reps, W=W, seed=23,
                                                         reads_per_warp=reads, group_of_sm=cg,
                                                         windows=cw)
+            # windows of the same size, evenly spaced and overlapping (policy 2)
+            ow, ocov = rr.rr_make_windows(N, W, S_w, groups.n_groups, policy=2)
+            covered, dmin, dmax = rr.rr_window_cover(ow, N // (128 * W))
+            rows[name]["overlapping"] = dict(
+                _stats(ses, N, reps, W=W, seed=23, reads_per_warp=reads,
+                       group_of_sm=groups.group_of_sm, windows=ow),
+                coverage=ocov, depth_min=dmin, depth_max=dmax)
         cfg4[f"{128 * W}B"] = {"unrestricted_full": _stats(ses, N, reps, W=W, seed=23,
                                                            reads_per_warp=reads),
                                "windows": rows}
@@ -246,6 +254,12 @@ def run(out_dir: Path, quick: bool = False) -> dict:
                                                  float(win[:, 1].max()) * 128 * W / GiB]}
     R["balanced_pooled"] = balanced
     R["seconds"] = time.time() - t_start
+    if alloc_study:
+        # the study maps the same amount of memory four ways: give the big buffer back first
+        del ses.buf
+        torch.cuda.empty_cache()
+        from . import alloc_study as study
+        R["alloc_study"] = study.run()
     (out_dir / "report.json").write_text(json.dumps(R, indent=1))
     (out_dir / "report.md").write_text(markdown(R))
     return R
@@ -298,11 +312,15 @@ def markdown(R: dict) -> str:
     L += ["", "## Grouped windows over the whole buffer", ""]
     for width, d in R["cfg4_grouped"].items():
         L += [f"### {width} lines: unrestricted over everything {f(d['unrestricted_full'])}", "",
-              "| window | GiB | coverage | grouped | unrestricted inside one window | naive per-SM |",
-              "|---|---|---|---|---|---|"]
+              "| window | GiB | coverage | grouped | unrestricted inside one window | naive per-SM "
+              "| overlapping windows (coverage, depth min-max) |",
+              "|---|---|---|---|---|---|---|"]
         for name, r in d["windows"].items():
+            o = r.get("overlapping")
+            ov = (f"{f(o)} ({o['coverage']:.2f}, {o['depth_min']}-{o['depth_max']})" if o else "")
             L.append(f"| {name} | {r['window_gib']:.1f} | {r['coverage']:.2f} | {f(r['grouped'])} | "
-                     f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} |")
+                     f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} "
+                     f"| {ov} |")
         L.append("")
     L += ["## One window per SM, windows spread over the buffer (equal work per SM)", "",
           "| window MiB | GB/s |", "|---|---|"]
@@ -326,6 +344,9 @@ def markdown(R: dict) -> str:
         L.append(f"| {name} | {b['burst_gbps']:.0f} | {b['sustained_gbps']:.0f} | "
                  f"{b['window_gib_min_max'][0]:.1f}-{b['window_gib_min_max'][1]:.1f} |")
     L.append("")
+    if "alloc_study" in R:
+        from . import alloc_study as study
+        L.append(study.markdown(R["alloc_study"]))
     L.append(f"total {R['seconds']:.0f} s")
     return "\n".join(L) + "\n"
 
@@ -334,8 +355,11 @@ def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default="report_out")
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--alloc-study", action="store_true",
+                    help="also map the same memory through four allocation paths and locate the "
+                         "cliff for each (Section 1.2: reach = translations x page size)")
     a = ap.parse_args(argv)
-    R = run(Path(a.out), a.quick)
+    R = run(Path(a.out), a.quick, a.alloc_study)
     print(markdown(R))
     return 0
 

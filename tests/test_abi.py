@@ -56,6 +56,19 @@ def test_read_argument_errors_come_before_any_cuda_call():
     assert _call(W=3) == rr.RR_ERR_ARG
     assert _call(mode=7) == rr.RR_ERR_ARG
     assert _call(index_mode=2) == rr.RR_ERR_ARG
+    assert _call(index_mode=4) == rr.RR_ERR_ARG
+    assert _call(index_mode=rr.RR_INDEX_MIXED) == rr.RR_ERR_ARG              # needs a period
+    assert _call(index_mode=rr.RR_INDEX_MIXED, mix_period=6) == rr.RR_ERR_ARG  # a power of two
+    assert _call(mix_period=4) == rr.RR_ERR_ARG                              # only with MIXED
+    srt = dict(variant=rr.RR_VARIANT_SORTED, sort_parts=4, sort_reads=64)
+    assert _call(**{**srt, "sort_parts": 3}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "sort_parts": 128}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "sort_reads": 48}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "sort_reads": 0}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "W": 4}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "index_mode": rr.RR_INDEX_STRIDE}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "unroll": 8}) == rr.RR_ERR_ARG
+    assert _call(sort_parts=4) == rr.RR_ERR_ARG                              # only with SORTED
     assert _call(variant=9) == rr.RR_ERR_ARG
     assert _call(unroll=3) == rr.RR_ERR_ARG
     assert _call(n_warps=0) == rr.RR_ERR_ARG
@@ -111,16 +124,19 @@ def test_other_entry_points_reject_bad_arguments():
 
 def test_make_windows_matches_oracle():
     for L, S, G, W, policy in itertools.product((1, 2, 7, 40, 1000, 12345), (1, 3, 64, 999, 10 ** 6),
-                                                (1, 2, 5, 14, 148), (1, 2, 4), (0, 1)):
+                                                (1, 2, 5, 14, 148), (1, 2, 4), (0, 1, 2)):
         lb = 128 * W
         a, ca = rr.rr_make_windows(L * lb + 5, W, S * lb, G, policy, seed=23)
         b, cb = oracle.make_windows(L * lb + 5, W, S * lb, G, policy, seed=23)
         assert np.array_equal(a, b) and ca == cb
     big = int(0.95 * 178 * (1 << 30)) // 512 * 512
     for S in (big // 8, big // 4, big // 2, big, 64 << 30, 37 << 30):
-        a, ca = rr.rr_make_windows(big, 1, S, 16)
-        b, cb = oracle.make_windows(big, 1, S, 16)
-        assert np.array_equal(a, b) and ca == cb
+        for policy in (0, 2):
+            a, ca = rr.rr_make_windows(big, 1, S, 16, policy)
+            b, cb = oracle.make_windows(big, 1, S, 16, policy)
+            assert np.array_equal(a, b) and ca == cb
+    with pytest.raises(rr.RRError):
+        rr.rr_make_windows(1 << 20, 1, 1 << 10, 2, policy=3)
     with pytest.raises(rr.RRError):
         rr.rr_make_windows(1 << 20, 3, 1 << 10, 2)
     with pytest.raises(rr.RRError):
@@ -201,6 +217,120 @@ def test_reach_matches_oracle():
         rr.rr_reach([2 << 30, 1 << 30], [1.0, 1.0])
     with pytest.raises(rr.RRError):
         rr.rr_reach([1 << 30], [1.0])
+
+
+def test_reach_next_and_sm_reach_match_oracle():
+    rng = np.random.default_rng(7)
+    GiB = 1 << 30
+    for _ in range(300):
+        sizes = sorted({int(x) * 2 * GiB for x in rng.integers(1, 85, int(rng.integers(3, 14)))})
+        if sizes[0] > 32 * GiB:
+            sizes = [4 * GiB] + sizes
+        g = rng.uniform(3000, 4600, len(sizes))
+        cut = int(rng.integers(1, len(sizes) + 1))
+        g[cut:] *= rng.choice([0.3, 0.85, 0.5])
+        step = int(rng.choice([1, 2, 4])) * GiB
+        try:
+            expect = oracle.reach_next(sizes, g, step)
+        except oracle.OracleError:
+            with pytest.raises(rr.RRError):
+                rr.rr_reach_next(sizes, g, step)
+            continue
+        assert rr.rr_reach_next(sizes, g, step) == expect
+    with pytest.raises(rr.RRError):
+        rr.rr_reach_next([4 * GiB, 8 * GiB], [1.0, 1.0], 0)
+    for _ in range(300):
+        n = int(rng.integers(1, 12))
+        sizes = np.cumsum(rng.integers(1, 300, n)).astype(np.uint64) << 20
+        rates = rng.uniform(4500, 6000, n)
+        keep = float(rng.choice([1.0, 0.99, 0.97, 0.9, 0.6]))
+        assert rr.rr_sm_reach(sizes, rates, keep) == oracle.sm_reach(sizes, rates, keep)
+    with pytest.raises(rr.RRError):
+        rr.rr_sm_reach([2, 2], [1.0, 1.0])
+    with pytest.raises(rr.RRError):
+        rr.rr_sm_reach([1, 2], [1.0, 1.0], keep=0.0)
+
+
+def test_owner_map_phase_window_and_cover_match_oracle():
+    rng = np.random.default_rng(8)
+    for _ in range(200):
+        nsm = int(rng.integers(1, 257))
+        g = rng.integers(0, int(rng.integers(1, 40)), nsm).astype(np.uint16)
+        g[rng.random(nsm) < 0.1] = 0xFFFF
+        a, na = rr.rr_owner_map(g)
+        b, nb = oracle.owner_map(g)
+        assert na == nb and np.array_equal(a, b)
+    for _ in range(500):
+        sl, reach = int(rng.integers(1, 1 << 36)), int(rng.integers(1, 1 << 32))
+        mp = int(rng.choice([1, 8, 64, 1000]))
+        assert rr.rr_phase_window(sl, reach, mp) == oracle.phase_window(sl, reach, mp)
+    with pytest.raises(rr.RRError):
+        rr.rr_phase_window(0, 1 << 20)
+    for _ in range(300):
+        L = int(rng.integers(1, 10 ** 6))
+        G = int(rng.integers(1, 60))
+        base = rng.integers(0, L, G)
+        n = np.minimum(rng.integers(1, L + 1, G), L - base)
+        win = np.stack([base, np.maximum(n, 1)], axis=1).astype(np.uint32)
+        win[:, 1] = np.minimum(win[:, 1], L - win[:, 0])
+        assert rr.rr_window_cover(win, L) == oracle.window_cover(win, L)
+    with pytest.raises(rr.RRError):
+        rr.rr_window_cover([[5, 10]], 12)
+
+
+def test_rebalance_and_spread_match_oracle():
+    rng = np.random.default_rng(9)
+    for _ in range(400):
+        G = int(rng.integers(1, 150))
+        work = rng.integers(0, 1 << int(rng.integers(1, 31)), G).astype(np.uint32)
+        fin = rng.integers(1, 1 << int(rng.integers(8, 45)), G).astype(np.uint64)
+        fin[rng.random(G) < 0.1] = 0
+        scale = int(rng.integers(1, 1 << 31))
+        assert rr.rr_finish_spread_ppm(fin) == oracle.finish_spread_ppm(fin)
+        try:
+            expect = oracle.rebalance_weights(work, fin, scale)
+        except oracle.OracleError:
+            with pytest.raises(rr.RRError):
+                rr.rr_rebalance_weights(work, fin, scale)
+            continue
+        assert np.array_equal(rr.rr_rebalance_weights(work, fin, scale), expect)
+
+
+def test_group_finish_matches_oracle():
+    rng = np.random.default_rng(11)
+    for _ in range(300):
+        nsm = int(rng.integers(1, 257))
+        G = int(rng.integers(1, 40))
+        g = rng.integers(0, G, nsm).astype(np.uint16)
+        g[rng.random(nsm) < 0.1] = 0xFFFF
+        t0 = rng.integers(1 << 40, (1 << 40) + 5000, nsm).astype(np.uint64)
+        t1 = t0 + rng.integers(1, 1 << 22, nsm).astype(np.uint64)
+        t1[rng.random(nsm) < 0.1] = 0
+        a, sa = rr.rr_group_finish(t0, t1, g, G)
+        b, sb = oracle.group_finish(t0, t1, g, G)
+        assert np.array_equal(a, b) and sa == sb
+    with pytest.raises(rr.RRError):
+        rr.rr_group_finish([1], [2], [3], 2)
+
+
+def test_probe_rate_matches_oracle():
+    rng = np.random.default_rng(10)
+    for _ in range(500):
+        t0 = rng.integers(1 << 40, 1 << 41, 2).astype(np.uint64)
+        t1 = t0 + rng.integers(0, 1 << 22, 2).astype(np.uint64)
+        claim = rng.integers(0, 3, 2).astype(np.uint32)
+        if rng.random() < 0.1:
+            t1[int(rng.integers(0, 2))] = 0
+        solo = bool(rng.random() < 0.3)
+        reads = int(rng.integers(1, 1 << 24)) * 2
+        try:
+            expect = oracle.probe_rate(t0, t1, claim, solo, reads)
+        except oracle.OracleError as e:
+            with pytest.raises(rr.RRError) as r:
+                rr.rr_probe_rate(t0, t1, claim, solo, reads)
+            assert r.value.code == e.code == rr.RR_ERR_SM_UNCOVERED
+            continue
+        assert rr.rr_probe_rate(t0, t1, claim, solo, reads) == expect
 
 
 def test_exact_remainder_identity():

@@ -278,3 +278,88 @@ def test_moving_window_over_all_of_memory_from_every_sm_sampled(ses):
         st = oracle.stagger_of_sm(v // WPS, ses.nsm, L, sub_bytes // 128)
         assert tuple(got[v]) == oracle.warp_checksum_phased(7, v, 0, reads, 1, 0, L, 1024,
                                                             sub_bytes // 128, st), v
+
+
+def test_session_helpers_run_the_plans_they_describe(ses):
+    """measure_group_rates, naive_control and windows(): the launches they make are the oracle's
+    (checksums, not rates)."""
+    groups = rr_inputs.synthetic_group_map(ses.nsm, 12, seed=5)
+    from paper_2405_11425_b200.pipeline import Groups
+    G = Groups(groups, 12, 10.0)
+    S = 16 * GiB
+    rates = ses.measure_group_rates(G, S, reads_per_warp=256)
+    assert len(rates) == 12 and all(r > 1 for r in rates)
+    # the last launch of measure_group_rates: group 11 alone inside [0, S)
+    only = np.where(groups == 11, 0, 0xFFFF).astype(np.uint16)
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), ses.region_bytes, 1, 256, 23, only,
+                   np.array([[0, S // 128]], np.uint32))
+    cg, cw, cov = ses.naive_control(S, 23)
+    assert 0 < cov <= 1 and cg.tolist() == list(range(ses.nsm))
+    ow, ocov = oracle.make_windows(ses.region_bytes, 1, S, ses.nsm, policy=1, seed=23)
+    assert np.array_equal(cw, ow) and cov == ocov
+    rate, res = ses.read(ses.region_bytes, seed=23, reads_per_warp=300, group_of_sm=cg, windows=cw)
+    assert res.sms_covered == ses.nsm
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), ses.region_bytes, 1, 300, 23, cg, cw)
+    win, cov = ses.windows(G, S)
+    ow, ocov = oracle.make_windows(ses.region_bytes, 1, S, 12)
+    assert np.array_equal(win, ow) and cov == ocov
+
+
+def test_sustained_protocol_reports_what_it_ran(ses):
+    p = ses.params(8 * GiB, seed=7, reads_per_warp=1024, variant=rr.RR_VARIANT_PACKED, unroll=2)
+    d = ses.sustained(p, settle=10, min_ms=20.0, reps=3)
+    assert d["regions"] == 3 and d["launches_per_region"] >= 1
+    assert d["bytes_per_launch"] == ses.nsm * WPS * 1024 * 128
+    assert d["gbps_min"] <= d["gbps"] <= d["gbps_max"] and d["gbps"] > 100
+    assert d["ms_per_region"] >= 15.0
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), 8 * GiB, 1, 1024, 7)
+
+
+def test_reach_measurement_refines_between_sweep_points(ses):
+    r = ses.measure_reach(sizes_gib=(4, 16, 32, 64, 96, 128), sustained=False)
+    sizes = [s for s, _ in r.sweep]
+    assert sizes == sorted(sizes) and len(set(sizes)) == len(sizes)
+    import oracle as orc
+    assert (r.cliff, r.plateau_gbps, r.reach_bytes) == orc.reach(sizes, [g for _, g in r.sweep])
+    if r.cliff:                                       # refined to the 2 GiB grid
+        above = min(s for s in sizes if s > r.reach_bytes)
+        assert above - r.reach_bytes <= 2 * GiB
+
+
+def test_probe_rows_and_checkpoint_resume(ses, tmp_path):
+    # rows probed block by block equal... not bit for bit (rates are measurements), but they fill
+    # exactly the rows asked for, and a resumed run keeps the finished rows untouched
+    reads = 2 * WPS * 64
+    T = np.zeros((ses.nsm, ses.nsm), np.float32)
+    st = rr.rr_probe_rows(ses.buf, 1 * GiB, reads, WPS, 5, 1, 10, 13, T, ses.probe_out,
+                          ses.probe_scratch)
+    touched = np.zeros_like(T, dtype=bool)
+    touched[10:13, 10:] = True
+    touched |= touched.T
+    assert (T[touched] > 0).all() and not T[~touched].any()
+    assert np.array_equal(T, T.T) and st["overlap_min"] <= 1.0
+    with pytest.raises(rr.RRError):
+        rr.rr_probe_rows(ses.buf, 1 * GiB, reads, WPS, 5, 1, 13, 13, T, ses.probe_out,
+                         ses.probe_scratch)
+    path = tmp_path / "probe.npz"
+    g1 = ses.discover_groups(probe_region_bytes=1 * GiB, total_reads=reads, repeats=1,
+                             checkpoint=path, rows_per_block=64)
+    with np.load(path) as z:
+        assert int(z["rows_done"]) == ses.nsm
+        saved = z["T"].copy()
+        meta, stats = str(z["meta"]), str(z["stats"])
+    assert np.array_equal(saved, g1.matrix) and (saved > 0).all()
+    # an interrupted run: only the first 64 rows done, marked with a value no probe produces
+    half = saved.copy()
+    half[64:, 64:] = 0
+    half[:64, :] = 12345.0
+    half[:, :64] = 12345.0
+    np.savez(path, T=half, rows_done=64, meta=meta, stats=stats)
+    g2 = ses.discover_groups(probe_region_bytes=1 * GiB, total_reads=reads, repeats=1,
+                             checkpoint=path, rows_per_block=64)
+    assert (g2.matrix[:64, :] == 12345.0).all() and (g2.matrix[:, :64] == 12345.0).all()
+    assert (g2.matrix[64:, 64:] > 0).all() and not (g2.matrix[64:, 64:] == 12345.0).any()
+    # other probe settings: the file is ignored and everything is probed afresh
+    g3 = ses.discover_groups(probe_region_bytes=1 * GiB, total_reads=reads, repeats=1, seed=6,
+                             checkpoint=path, rows_per_block=64)
+    assert not (g3.matrix == 12345.0).any()

@@ -16,16 +16,16 @@ def dev():
     import torch
     rr_build.build()
     torch.cuda.set_device(0)
-    info = rr.rr_device_info()
 
     class Dev:
         pass
 
     d = Dev()
     d.torch = torch
+    d.scratch = torch.zeros(rr.rr_scratch_bytes(), dtype=torch.uint8, device="cuda")
+    info = rr.rr_device_info(d.scratch)
     d.info = info
     d.nsm = info["nsm_prop"]
-    d.scratch = torch.zeros(rr.rr_scratch_bytes(), dtype=torch.uint8, device="cuda")
     d.buf_bytes = 1 << 30
     d.buf = torch.empty(d.buf_bytes, dtype=torch.uint8, device="cuda")
     assert d.buf.data_ptr() % 512 == 0
@@ -47,6 +47,7 @@ def test_device_facts(dev):
     assert i["cc_major"] == 10
     assert i["nsm_reg"] == i["nsm_prop"] <= rr.RR_MAX_SM
     assert i["theoretical_gbps"] > 1000 and i["total_bytes"] > 100 << 30
+    assert rr.rr_device_info()["nsm_reg"] == 0          # no scratch: nothing launched, not read
 
 
 @pytest.mark.parametrize("n_words", [0, 1, 3, 4, 5, 127, 1023, 1024, (1 << 20) + 3, 37 * 148 * 2048 + 2])
@@ -208,10 +209,36 @@ def test_probe_matrix_is_symmetric_and_positive(dev):
     scratch = dev.torch.zeros(rr.rr_probe_matrix_scratch_bytes(dev.nsm), dtype=dev.torch.uint8,
                               device="cuda")
     out = _out(dev, 2 * wps)
-    T, overlap = rr.rr_probe_matrix(dev.buf, dev.buf_bytes, 2 * wps * 64, wps, 5, 1, dev.nsm, out,
-                                    scratch)
+    T, stats, ov = rr.rr_probe_matrix(dev.buf, dev.buf_bytes, 2 * wps * 256, wps, 5, 1, dev.nsm,
+                                      out, scratch, with_overlaps=True)
     assert T.shape == (dev.nsm, dev.nsm) and np.array_equal(T, T.T)
     assert np.isfinite(T).all() and (T > 0).all()
+    # the overlap rule: every pair either ran side by side for 98 % of its measurement or is
+    # counted, and the count agrees with the per-pair matrix
+    assert np.array_equal(ov, ov.T) and (np.diag(ov) == 1).all()
+    low = int((ov[np.triu_indices(dev.nsm, 1)] < np.float32(0.98)).sum())
+    assert stats["pairs_below_goal"] == low
+    assert stats["overlap_min"] >= 0.98 or low > 0
+    assert abs(stats["overlap_min"] - float(ov.min())) < 1e-6
+    assert stats["reruns"] >= low                      # each of them was measured again at least once
+
+
+@pytest.mark.parametrize("W", [1, 2])
+def test_overlapping_windows_policy_on_gpu(dev, W):
+    """Policy 2: evenly spaced windows that overlap; warps of different groups may share lines."""
+    region = dev.buf_bytes
+    G = 7
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=3, inactive_frac=0.05)
+    windows, cov = rr.rr_make_windows(region, W, region // 4, G, policy=2)
+    assert cov == 1.0 and int(windows[-1].sum()) == region // (128 * W)
+    covered, dmin, dmax = rr.rr_window_cover(windows, region // (128 * W))
+    assert covered == region // (128 * W) and dmin >= 1 and dmax >= 2
+    out = _out(dev, dev.nsm * 8)
+    p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=8, reads_per_warp=77, seed=23,
+                      group_of_sm=groups, windows=windows, variant=rr.RR_VARIANT_PACKED, unroll=2)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_per_sm(region, W, dev.nsm, 8, 77, 23,
+                                                       group_of_sm=groups, windows=windows))
 
 
 @pytest.mark.parametrize("sizes,drop", [
@@ -457,3 +484,76 @@ def test_launch_configuration_is_cached(dev):
     assert {k: mid[k] for k in ("event_creates", "device_fact_queries")} == \
            {k: before[k] for k in ("event_creates", "device_fact_queries")}
     assert after == mid
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+@pytest.mark.parametrize("variant", [rr.RR_VARIANT_LDG, rr.RR_VARIANT_PACKED])
+def test_mixed_index_mode_matches_oracle(dev, W, variant):
+    region = dev.buf_bytes
+    G = 5
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=8, inactive_frac=0.05)
+    windows, _ = rr.rr_make_windows(region, W, region // 5, G)
+    windows[1] = (777, 10007)
+    for k, reads, first in [(1, 70, 0), (2, 133, 5), (8, 300, 64), (64, 257, 1000)]:
+        out = _out(dev, dev.nsm * 8)
+        p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=8, reads_per_warp=reads,
+                          first_read=first, seed=23, group_of_sm=groups, windows=windows,
+                          variant=variant, index_mode=rr.RR_INDEX_MIXED, mix_period=k)
+        rr.rr_random_read(p, out, dev.scratch)
+        expect = oracle.read_per_sm_mixed(region, W, dev.nsm, 8, reads, 23, k, group_of_sm=groups,
+                                          windows=windows, first_read=first)
+        assert np.array_equal(_np(out), expect), (W, variant, k, reads, first)
+    L = region // (128 * W)
+    out = _out(dev, 100)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=100, reads_per_warp=90,
+                      seed=3, variant=variant, index_mode=rr.RR_INDEX_MIXED, mix_period=4)
+    rr.rr_random_read(p, out, dev.scratch)
+    got = _np(out)
+    for v in range(0, 100, 7):
+        assert tuple(got[v]) == oracle.warp_checksum_mixed(3, v, 0, 90, W, 0, L, 4, n_warps_total=100)
+
+
+@pytest.mark.parametrize("W", [1, 2])
+@pytest.mark.parametrize("unroll", [0, 1, 4])
+@pytest.mark.parametrize("parts,sreads", [(2, 32), (4, 64), (8, 1024), (64, 32)])
+def test_sorted_variant_reads_the_same_lines_in_another_order(dev, W, unroll, parts, sreads):
+    """RR_VARIANT_SORTED only reorders a warp's reads (part by part of its window, epoch by epoch):
+    the checksums must be those of the plain definition, for every ragged length."""
+    region = 777 * MiB + 384
+    for reads, first in [(0, 0), (1, 0), (5, 3), (31, 0), (32, 1), (33, 0), (64, 0), (100, 7),
+                         (parts * sreads, 0), (parts * sreads + 1, 2), (3 * parts * sreads - 7, 5),
+                         (257, 2)]:
+        n_warps = 150
+        out = _out(dev, n_warps)
+        p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
+                          reads_per_warp=reads, first_read=first, seed=11, unroll=unroll,
+                          variant=rr.RR_VARIANT_SORTED, sort_parts=parts, sort_reads=sreads)
+        rr.rr_random_read(p, out, dev.scratch)
+        expect = oracle.read_logical(region, W, n_warps, reads, 11, first_read=first)
+        assert np.array_equal(_np(out), expect), (W, unroll, parts, sreads, reads, first)
+
+
+@pytest.mark.parametrize("W", [1, 2])
+def test_sorted_variant_grouped_and_pooled(dev, W):
+    region = dev.buf_bytes
+    G = 6
+    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=2, inactive_frac=0.05)
+    windows, _ = rr.rr_make_windows(region, W, region // 4, G)
+    windows[2] = (123, 3)                           # fewer lines than parts: some parts are empty
+    windows[4] = (5000, 1001)
+    kw = dict(variant=rr.RR_VARIANT_SORTED, sort_parts=4, sort_reads=64)
+    out = _out(dev, dev.nsm * 32)
+    p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=32, reads_per_warp=700, first_read=96,
+                      seed=23, group_of_sm=groups, windows=windows, **kw)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    assert res.sms_covered == int((groups != 0xFFFF).sum())
+    assert np.array_equal(_np(out), oracle.read_per_sm(region, W, dev.nsm, 32, 700, 23,
+                                                       group_of_sm=groups, windows=windows,
+                                                       first_read=96))
+    win, ws = rr.rr_make_weighted_windows(region, W, [3, 1, 2, 2, 5, 1], 999)
+    out = _out(dev, 999)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_POOLED, n_warps=999, warps_per_sm=32,
+                      nsm=dev.nsm, reads_per_warp=901, seed=5, group_of_sm=groups, windows=win,
+                      warp_start=ws, **kw)
+    rr.rr_random_read(p, out, dev.scratch)
+    assert np.array_equal(_np(out), oracle.read_pooled(region, W, win, ws, 901, 5))

@@ -88,3 +88,17 @@ def test_cfg0_batch_matches_kats(golden_dir):
     assert tuple(out[1]) == (0x64D363B4, 0x790CA7EE)
     assert tuple(out[2]) == (0x5AF2F0EC, 0x11B53B6C)
     assert tuple(out[65535]) == (0xA8E997CD, 0xE4F3550B)
+
+
+def test_golden_file_is_what_the_definitions_give(golden_dir):
+    # the committed known answers are regenerated, byte for byte, by a script that uses Python
+    # integers only and imports nothing of this repository
+    import subprocess
+    import sys
+    import re
+    src = (golden_dir / "derive_kats.py").read_text()
+    imported = set(re.findall(r"^\s*(?:import|from)\s+([\w.]+)", src, flags=re.M))
+    assert imported == {"__future__", "sys", "pathlib"}
+    r = subprocess.run([sys.executable, str(golden_dir / "derive_kats.py"), "--check"],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr

@@ -10,8 +10,9 @@ import torch.multiprocessing as mp
 
 import numpy as np
 
-from paper_2405_11425_b200.pipeline import (Groups, Reach, aggregate_throughput, finish_spread,
-                                             load_calibration, rebalanced_weights,
+from paper_2405_11425_b200.binding import RRError, rr_finish_spread_ppm
+from paper_2405_11425_b200.binding import rr_rebalance_weights as rebalanced_weights
+from paper_2405_11425_b200.pipeline import (Groups, Reach, aggregate_throughput, load_calibration,
                                              save_calibration)
 
 
@@ -55,18 +56,18 @@ def test_single_process_is_identity():
 def test_rebalancing_moves_work_towards_groups_that_finished_early():
     # three groups with true capacities 2 : 1 : 1 given equal work: the first finishes in half
     # the time; one update makes the weights proportional to the capacities
-    w = rebalanced_weights([100, 100, 100], [500.0, 1000.0, 1000.0])
+    w = rebalanced_weights([100, 100, 100], [500, 1000, 1000])
     assert w.sum() in range(999_990, 1_000_010)
     assert abs(w[0] / w[1] - 2.0) < 1e-3 and w[1] == w[2]
     # a fixed point: work already proportional to capacity -> same finish -> same weights
-    w2 = rebalanced_weights(w, [7.0, 7.0, 7.0])
-    assert np.array_equal(w, w2)
+    w2 = rebalanced_weights(w, [7000, 7000, 7000])
+    assert np.abs(w.astype(np.int64) - w2.astype(np.int64)).max() <= 1
     # a group that never ran keeps a token weight, never zero
-    w3 = rebalanced_weights([100, 100], [1000.0, 0.0])
+    w3 = rebalanced_weights([100, 100], [1000, 0])
     assert w3[1] >= 1 and w3[0] > 100 * w3[1]
-    assert finish_spread([1000.0, 980.0, 0.0]) == pytest.approx(0.02)
-    with pytest.raises(ValueError):
-        rebalanced_weights([1, 1], [0.0, 0.0])
+    assert rr_finish_spread_ppm([1000, 980, 0]) == 20_000
+    with pytest.raises(RRError):
+        rebalanced_weights([1, 1], [0, 0])
 
 
 def test_calibration_round_trip_is_bound_to_the_card(tmp_path):
