@@ -53,6 +53,7 @@ ITERS_PER_ARM_LAUNCH = 64     # the arms queue shorter launches back to back
 WARPS_PER_SM = 32
 SETTLE_LAUNCHES = 150         # of the same launch, before any timed region
 VARIANT_PACKED = 2            # 16-byte lanes: one warp load covers four 128-byte lines
+VARIANT_SORTED = 3            # the same, each warp's reads taken part by part of its window
 UNROLL = 2                    # warp loads in flight per warp (8 lines)
 SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
@@ -289,6 +290,13 @@ def run_gpu(args):
         window_gib_min_max=[N / GiB, N / GiB], coverage=1.0,
         sub_window_mib=mv_sub / (1 << 20), phase_reads=1024,
         note="every SM's window is the whole buffer; SM cycles staggered")
+    # static per-SM slices, equal work, no calibration of weights: the kernel performs each warp's
+    # reads part by part of its window (same reads and checksums, another order)
+    arms["g_sorted_execution_static_per_sm_slices"] = measure(
+        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
+                   windows=mv_windows, variant=VARIANT_SORTED, unroll=1, sort_parts=4,
+                   sort_reads=1024), mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
+        kernel="read_kernel<U=1, sorted>")
     t_arms = time.time() - t_arms
     c_head = cfg4[headline]["gbps"]
     comparison = {
@@ -458,7 +466,7 @@ def run_gpu(args):
             "arms": arms,
             "protocol": {"settle_launches": SETTLE_LAUNCHES, "min_ms_per_region": 50.0,
                          "regions": 5, "reads_per_warp_per_launch": arm_reads,
-                         "kernel": "read_kernel<U=2, packed> for every arm",
+                         "kernel": "read_kernel<U=2, packed> for every arm but g",
                          "seconds_all_arms": t_arms},
             "calibration": {
                 "device": ses.info["name"], "uuid": ses.info["uuid"], "nsm": ses.nsm,

@@ -76,11 +76,7 @@ extern "C" {
 #define RR_VARIANT_LDG_CHECKED 1u /* same, every address bounds-checked before the load         */
 #define RR_VARIANT_PACKED 2u      /* every lane loads 16 bytes: one warp load covers 4/W lines  */
                                   /* (same lines and words; fewer instructions per line)        */
-#define RR_VARIANT_L2_128 3u      /* RR_VARIANT_LDG with the .L2::128B prefetch qualifier       */
-#define RR_VARIANT_L2_256 4u      /* RR_VARIANT_LDG with the .L2::256B prefetch qualifier       */
-#define RR_VARIANT_BULK 5u        /* one cp.async.bulk per line into a ring in shared memory,   */
-                                  /* completion on an mbarrier, lanes fold from shared memory   */
-#define RR_VARIANT_SORTED 6u      /* RR_VARIANT_PACKED with each warp's reads taken in an order */
+#define RR_VARIANT_SORTED 3u      /* RR_VARIANT_PACKED with each warp's reads taken in an order */
                                   /* that keeps the SM inside one part of its window at a time  */
 
 const char *rr_strerror(int32_t code);
@@ -298,8 +294,8 @@ size_t rr_probe_matrix_scratch_bytes(uint32_t nsm);
  * `repeats` sweeps, repeats >= 1), T_host[a*nsm+a] = solo GB/s.  Launches are queued back to
  * back per sweep and read back once.  out_dev as in rr_probe_pair (overwritten by every pair).
  *
- * The two SMs of a pair must read side by side for the figure to mean contention, so (i) the
- * first of the two blocks to arrive waits (at most 0.2 ms) for the other before it starts, and
+ * The two SMs of a pair must read side by side for the figure to mean contention, so (i) they
+ * start together and read until both are done (see rr_probe_pair), and
  * (ii) a pair whose overlap fraction
  *   (earliest end - latest start) / (latest end - earliest start)
  * is below 0.98 is measured again on its own with twice the reads, up to three doublings and
@@ -330,14 +326,14 @@ int32_t rr_probe_rows(const void *buf /*DEVICE*/, uint64_t region_bytes, uint64_
                       void *out_dev /*DEVICE*/, void *scratch_dev /*DEVICE*/,
                       rr_probe_stats_t *stats /*HOST*/, float *overlap_host /*HOST*/, void *stream);
 
-/* The rule that turns one probe's timers into a rate (host only).  t_start, t_end (ns) and claim
- * hold one entry per SM (two for a pair, the first only when solo = 1); an SM with claim 0 or
- * no end time never ran: RR_ERR_SM_UNCOVERED.  gbps = bytes of the SMs that ran (total_reads/2
- * lines of 128 bytes each) / (latest end - earliest start); overlap as defined above (1 for a
- * solo run).                                                                                  */
+/* The rule that turns one probe's timers into a rate (host only).  t_start, t_end (ns), claim and
+ * extra_lines hold one entry per SM (two for a pair, the first only when solo = 1); an SM with
+ * claim 0 or no end time never ran: RR_ERR_SM_UNCOVERED.  gbps = bytes of the SMs that ran
+ * (total_reads/2 + extra_lines[i] lines of 128 bytes each) / (latest end - earliest start);
+ * overlap as defined above (1 for a solo run).                                                */
 int32_t rr_probe_rate(const uint64_t *t_start, const uint64_t *t_end, const uint32_t *claim,
-                      uint32_t solo, uint64_t total_reads, double *gbps, double *seconds,
-                      double *overlap);
+                      const uint64_t *extra_lines, uint32_t solo, uint64_t total_reads,
+                      double *gbps, double *seconds, double *overlap);
 
 /* ---- contention matrix -> SM groups --------------------------------------------------------
  * Paper, Section 2.2 and Figure 3 (the SM indices are reordered until the groups show up as

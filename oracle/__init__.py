@@ -107,7 +107,7 @@ def _load():
         lib.orc_window_cover.restype = i32
         lib.orc_window_cover.argtypes = [p, p, u32, u64, p, p, p]
         lib.orc_probe_rate.restype = i32
-        lib.orc_probe_rate.argtypes = [p, p, p, u32, u64, p, p, p]
+        lib.orc_probe_rate.argtypes = [p, p, p, p, u32, u64, p, p, p]
         _lib = lib
     return _lib
 
@@ -451,15 +451,16 @@ def window_cover(windows, n_lines: int):
     return int(cov.value), int(lo.value), int(hi.value)
 
 
-def probe_rate(t_start, t_end, claim, solo: bool, total_reads: int):
+def probe_rate(t_start, t_end, claim, solo: bool, total_reads: int, extra_lines=(0, 0)):
     """(GB/s, seconds, overlap) of one probe from its timers; OracleError(-6) if an SM never ran."""
     a = np.ascontiguousarray(t_start, dtype=np.uint64)
     b = np.ascontiguousarray(t_end, dtype=np.uint64)
     c = np.ascontiguousarray(claim, dtype=np.uint32)
+    x = np.ascontiguousarray(extra_lines, dtype=np.uint64)
     g = ctypes.c_double()
     sec = ctypes.c_double()
     ov = ctypes.c_double()
-    rc = _load().orc_probe_rate(_ptr(a), _ptr(b), _ptr(c), 1 if solo else 0, total_reads,
+    rc = _load().orc_probe_rate(_ptr(a), _ptr(b), _ptr(c), _ptr(x), 1 if solo else 0, total_reads,
                                 ctypes.byref(g), ctypes.byref(sec), ctypes.byref(ov))
     if rc != 0:
         raise OracleError(rc)

@@ -980,30 +980,37 @@ int32_t orc_finish_spread_ppm(const uint64_t *finish_ns, uint32_t n_groups, uint
 }
 
 /* ---- O11: rate and overlap of one two-SM probe (Section 2.2, Fig. 2) --------------------
- * Each chosen SM performs total_reads / 2 line reads of 128 bytes.  The pair's throughput
- * counts the bytes of both SMs over the union of their two intervals,
+ * Each chosen SM performs total_reads / 2 line reads of 128 bytes (the part whose checksums
+ * are verified) and then keeps reading until the other SM has finished its own share, so
+ * that two SMs of different speed still run side by side for the whole measurement;
+ * extra_lines[i] counts what SM i read beyond its share.  The pair's throughput counts every
+ * line read by both SMs over the union of their two intervals,
  *   GB/s = bytes / (latest end - earliest start)        (timers in ns, so bytes/ns = GB/s)
  * and the figure only means contention if the two ran side by side:
  *   overlap = (earliest end - latest start) / (latest end - earliest start), 0 if disjoint.
- * A solo run (one SM) has overlap 1.  An SM that claimed nothing or never ended: -6.     */
+ * A solo run (one SM) has overlap 1 and no extra lines.  An SM that claimed nothing or never
+ * ended: -6.                                                                            */
 #define ORC_ERR_SM_UNCOVERED (-6)
 int32_t orc_probe_rate(const uint64_t *t_start, const uint64_t *t_end, const uint32_t *claim,
-                       uint32_t solo, uint64_t total_reads, double *gbps, double *seconds,
-                       double *overlap)
+                       const uint64_t *extra_lines, uint32_t solo, uint64_t total_reads,
+                       double *gbps, double *seconds, double *overlap)
 {
-    if (!t_start || !t_end || !claim || !gbps || !seconds || !overlap || solo > 1) return ORC_ERR_ARG;
+    if (!t_start || !t_end || !claim || !extra_lines || !gbps || !seconds || !overlap || solo > 1)
+        return ORC_ERR_ARG;
     uint32_t k = solo ? 1 : 2;
     for (uint32_t i = 0; i < k; ++i)
         if (claim[i] == 0 || t_end[i] == 0 || t_end[i] < t_start[i]) return ORC_ERR_SM_UNCOVERED;
     uint64_t s_lo = t_start[0], s_hi = t_start[0], e_lo = t_end[0], e_hi = t_end[0];
+    uint64_t lines = total_reads / 2 + extra_lines[0];
     if (k == 2) {
         if (t_start[1] < s_lo) s_lo = t_start[1];
         if (t_start[1] > s_hi) s_hi = t_start[1];
         if (t_end[1] < e_lo) e_lo = t_end[1];
         if (t_end[1] > e_hi) e_hi = t_end[1];
+        lines += total_reads / 2 + extra_lines[1];
     }
     uint64_t span = e_hi - s_lo;
-    uint64_t bytes = (total_reads / 2) * k * 128ull;
+    uint64_t bytes = lines * 128ull;
     *seconds = (double)span * 1e-9;
     *gbps = span ? (double)bytes / (double)span : 0.0;
     *overlap = (span && e_lo > s_hi) ? (double)(e_lo - s_hi) / (double)span : 0.0;

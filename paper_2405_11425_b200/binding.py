@@ -24,7 +24,7 @@ RR_MAX_SM, RR_MAX_GROUPS, RR_MAX_WARPS_PER_SM, RR_SM_INACTIVE = 256, 256, 32, 0x
 RR_MODE_LOGICAL, RR_MODE_PER_SM, RR_MODE_POOLED = 0, 1, 2
 RR_INDEX_RANDOM, RR_INDEX_STRIDE, RR_INDEX_PHASED, RR_INDEX_MIXED = 0, 1, 2, 3
 RR_VARIANT_LDG, RR_VARIANT_LDG_CHECKED, RR_VARIANT_PACKED = 0, 1, 2
-RR_VARIANT_L2_128, RR_VARIANT_L2_256, RR_VARIANT_BULK, RR_VARIANT_SORTED = 3, 4, 5, 6
+RR_VARIANT_SORTED = 3
 
 EXPORTS = (
     "rr_strerror", "rr_last_cuda_error", "rr_device_info", "rr_scratch_bytes", "rr_fill",
@@ -145,7 +145,7 @@ def _load():
     lib.rr_probe_rows.restype = i32
     lib.rr_probe_rows.argtypes = [p, u64, u64, u32, u64, u32, u32, u32, p, u32, p, p, p, p, p]
     lib.rr_probe_rate.restype = i32
-    lib.rr_probe_rate.argtypes = [p, p, p, u32, u64, p, p, p]
+    lib.rr_probe_rate.argtypes = [p, p, p, p, u32, u64, p, p, p]
     lib.rr_reach_next.restype = i32
     lib.rr_reach_next.argtypes = [p, p, u32, u64, p]
     lib.rr_sm_reach.restype = i32
@@ -358,15 +358,16 @@ def rr_probe_rows(buf, region_bytes: int, total_reads: int, warps_per_sm: int, s
             "reruns": int(st.reruns), "relaunched": int(st.relaunched)}
 
 
-def rr_probe_rate(t_start, t_end, claim, solo: bool, total_reads: int):
+def rr_probe_rate(t_start, t_end, claim, solo: bool, total_reads: int, extra_lines=(0, 0)):
     """(GB/s, seconds, overlap) of one probe from its timers (host rule, no GPU involved)."""
     a = np.ascontiguousarray(t_start, dtype=np.uint64)
     b = np.ascontiguousarray(t_end, dtype=np.uint64)
     c = np.ascontiguousarray(claim, dtype=np.uint32)
+    x = np.ascontiguousarray(extra_lines, dtype=np.uint64)
     g, sec, ov = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
-    _check(_load().rr_probe_rate(a.ctypes.data, b.ctypes.data, c.ctypes.data, 1 if solo else 0,
-                                 total_reads, ctypes.byref(g), ctypes.byref(sec), ctypes.byref(ov)),
-           "rr_probe_rate")
+    _check(_load().rr_probe_rate(a.ctypes.data, b.ctypes.data, c.ctypes.data, x.ctypes.data,
+                                 1 if solo else 0, total_reads, ctypes.byref(g), ctypes.byref(sec),
+                                 ctypes.byref(ov)), "rr_probe_rate")
     return float(g.value), float(sec.value), float(ov.value)
 
 

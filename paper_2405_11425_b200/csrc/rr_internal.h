@@ -25,7 +25,12 @@ struct ProbeRecord {      // one per probe launch
     uint32_t claim[2];
     uint32_t ready;       // chosen SMs that have arrived at the common start
     uint32_t gave_up;     // chosen SMs that stopped waiting for the other one
+    uint32_t done_warps[2];            // warps of each SM that have finished their fixed share
+    unsigned long long extra_lines[2]; // lines each SM read beyond its share, waiting for the other
+    uint32_t sink;        // never read: keeps the extra loads observable
+    uint32_t pad;
 };
+static_assert(sizeof(ProbeRecord) % 16 == 0, "records are packed in an array");
 
 struct ScratchHeader {
     uint32_t status;

@@ -96,22 +96,15 @@ struct ReadArgs {
     ScratchHeader *scratch;
 };
 
-constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarL2_128 = 3, kVarL2_256 = 4,
-              kVarBulk = 5, kVarSorted = 6;
-__host__ __device__ constexpr int l2_hint_of(int var) { return var == kVarL2_128 ? 128 : (var == kVarL2_256 ? 256 : 0); }
+constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarSorted = 3;
 
-// Per-warp state of the bulk-copy shape: a ring of U line slots and U mbarriers in shared memory
-// (32-bit shared-window addresses), and the phase parity each barrier will complete next.
-struct BulkRing {
-    uint32_t ring, bars, phases;
-    uint32_t *status;
+// Per-warp working memory some variants need beside their registers.
+struct WarpScratch {
     uint32_t *queue;  // SORTED variant: this warp's ring of kSortQueue line indices (shared memory)
 };
 constexpr uint32_t kSortQueue = 64;  // two vectors of 32 lines
-constexpr uint32_t kBulkWaitPolls = 1u << 20;  // per line; each poll may itself sleep a little
-constexpr uint32_t kStatusBulkTimeout = 2u;    // status bit: a bulk copy did not complete in time
 
-template <int W, int U, bool CHECKED, int HINT>
+template <int W, int U, bool CHECKED>
 __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, uint64_t region_bytes,
                                            uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
@@ -140,7 +133,7 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
                 return;
             }
         }
-        load_lane<W, HINT>(lane_ptr + (uint64_t)line * (128u * W), dst);
+        load_lane<W>(lane_ptr + (uint64_t)line * (128u * W), dst);
     };
     auto fold = [&](const uint32_t(&src)[W]) {
 #pragma unroll
@@ -348,7 +341,7 @@ template <int W, int U>
 __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, uint64_t key,
                                                   IndexSpec ix, uint64_t first, uint64_t reads,
                                                   uint32_t base, uint32_t n, uint32_t lane,
-                                                  uint32_t &X, uint32_t &S, BulkRing &br)
+                                                  uint32_t &X, uint32_t &S, WarpScratch &br)
 {
     constexpr int P = 4 / W;     // lines per warp load
     constexpr int NL = 32 / P;   // warp loads per vector of 32 lines = lanes per line
@@ -412,140 +405,31 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
     S = s;
 }
 
-// Bulk-copy shape: lane 0 asks the copy engine for each whole line (cp.async.bulk into the warp's
-// ring in shared memory, completion counted on an mbarrier), the lanes then fold the line from
-// shared memory.  One request per line instead of 32 lane requests; same lines, same words.
-// Every wait is bounded: a copy that does not complete sets kStatusBulkTimeout, the warp stops
-// issuing, waits (bounded again) for what is still in flight and returns what it has.
-template <int W, int U>
-__device__ __forceinline__ void warp_reads_bulk(const char *__restrict__ buf, uint64_t key,
-                                                IndexSpec ix, uint64_t v, uint64_t V,
-                                                uint64_t first, uint64_t reads, uint32_t base,
-                                                uint32_t n, uint32_t lane, uint32_t &X, uint32_t &S,
-                                                BulkRing &br)
-{
-    static_assert(U >= 1 && U <= 16 && (32 % U) == 0, "ring depth must divide a batch");
-    constexpr uint32_t kLine = 128u * W;
-    LineSource src;
-    src.init(base, n, ix);
-    uint32_t x = 0, s = 0;
-    uint32_t inflight = 0;  // slots with a copy in flight (warp-uniform)
-    bool dead = false;      // a wait ran out (warp-uniform)
-
-    auto gen = [&](uint64_t i) -> uint32_t {
-        const uint64_t r = draw_index(ix, key, i, v, V);
-        return src.base + mod_exact(r, src.div);
-    };
-    auto issue = [&](uint32_t line, int slot) {
-        if (lane == 0) {
-            const uint32_t bar = br.bars + 8u * slot;
-            mbar_expect_tx(bar, kLine);
-            bulk_load(br.ring + kLine * slot, buf + (uint64_t)line * kLine, kLine, bar);
-        }
-        inflight |= 1u << slot;
-    };
-    auto wait = [&](int slot) -> bool {
-        const uint32_t bar = br.bars + 8u * slot, parity = (br.phases >> slot) & 1u;
-        bool ok = false;
-        for (uint32_t k = 0; k < kBulkWaitPolls && !ok; ++k) ok = mbar_try_wait(bar, parity);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        br.phases ^= 1u << slot;  // the barrier is left to its fate if the wait ran out
-        inflight &= ~(1u << slot);
-        return ok;
-    };
-    auto consume = [&](int slot) {
-        if (!wait(slot)) {
-            dead = true;
-            if (lane == 0) atomicOr(br.status, kStatusBulkTimeout);
-            return;
-        }
-        uint32_t d[W];
-        lds_lane(br.ring + kLine * slot + lane * (4u * W), d);
-#pragma unroll
-        for (int w = 0; w < W; ++w) {
-            x ^= d[w];
-            s += d[w];
-        }
-    };
-
-    const uint64_t n_batches = (reads + 31) >> 5;
-    src.enter(first, ix);
-    uint32_t cur = gen(first + lane);
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u);
-        if ((uint64_t)u < reads) issue(line, u);
-    }
-    for (uint64_t b = 0; b < n_batches; ++b) {
-        const uint64_t t0 = b << 5;
-        src.enter(first + t0 + 32, ix);
-        const uint32_t nxt = gen(first + t0 + 32 + lane);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const uint64_t t = t0 + j;
-            if (t < reads && !dead) consume(j % U);
-            uint32_t line = (j + U < 32) ? __shfl_sync(0xFFFFFFFFu, cur, (j + U) & 31)
-                                         : __shfl_sync(0xFFFFFFFFu, nxt, (j + U) & 31);
-            __syncwarp();  // every lane has read the slot before the copy engine may overwrite it
-            if (t + U < reads && !dead) issue(line, j % U);
-        }
-        cur = nxt;
-        if (dead) break;
-    }
-    if (dead)  // bounded wait for the copies still in flight: shared memory must outlive them
-        for (int u = 0; u < U; ++u)
-            if (inflight & (1u << u)) wait(u);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        x ^= __shfl_xor_sync(0xFFFFFFFFu, x, o);
-        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-    }
-    X = x;
-    S = s;
-}
-
 template <int W, int U, int VAR>
 __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_t region_bytes,
                                            uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
-                                           uint32_t &S, uint32_t *violations, BulkRing &br)
+                                           uint32_t &S, uint32_t *violations, WarpScratch &br)
 {
     if constexpr (VAR == kVarPacked && W < 4)
         warp_reads_packed<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S);
     else if constexpr (VAR == kVarSorted && W < 4)
         warp_reads_sorted<W, U>(buf, key, ix, first, reads, base, n, lane, X, S, br);
-    else if constexpr (VAR == kVarBulk)
-        warp_reads_bulk<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S, br);
     else
-        warp_reads_lines<W, U, VAR == kVarChecked, l2_hint_of(VAR)>(
-            buf, region_bytes, key, ix, v, V, first, reads, base, n, lane, X, S, violations);
+        warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, ix, v, V, first, reads,
+                                                   base, n, lane, X, S, violations);
 }
 
-// Dynamic shared memory: ballast that keeps one block per SM, and the bulk shape's rings.
-extern __shared__ __align__(128) unsigned char rr_dyn_smem[];
-
-template <int W, int U, int VAR>
-__device__ __forceinline__ BulkRing make_bulk_ring(uint32_t warp, uint32_t lane, uint32_t wpc,
-                                                   uint32_t *status)
+template <int VAR>
+__device__ __forceinline__ WarpScratch make_warp_scratch(uint32_t warp)
 {
-    BulkRing br{0u, 0u, 0u, status, nullptr};
+    WarpScratch ws{nullptr};
     if constexpr (VAR == kVarSorted) {
         __shared__ uint32_t sh_sort_queue[32 * kSortQueue];
-        br.queue = sh_sort_queue + warp * kSortQueue;
+        ws.queue = sh_sort_queue + warp * kSortQueue;
     }
-    if constexpr (VAR == kVarBulk) {
-        const uint32_t base = smem_addr(rr_dyn_smem);
-        br.ring = base + warp * (U * 128u * W);
-        br.bars = base + wpc * (U * 128u * W) + warp * (U * 8u);
-        if (lane == 0) {
-            for (int u = 0; u < U; ++u) mbar_init(br.bars + 8u * u, 1u);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
-        __syncwarp();
-    }
-    return br;
+    return ws;
 }
 
 template <int W, int U, int VAR>
@@ -557,7 +441,7 @@ __global__ void __launch_bounds__(1024, 1)
     __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     ScratchHeader *sc = a.scratch;
-    BulkRing br = make_bulk_ring<W, U, VAR>(warp, lane, a.wpc, &sc->status);
+    WarpScratch br = make_warp_scratch<VAR>(warp);
 
     if (a.mode == RR_MODE_POOLED) {
         // Work sharing inside an SM group: items (logical warp, block of reads) come from the
@@ -714,6 +598,7 @@ struct ProbeArgs {
 constexpr int kProbeUnroll = 8;
 constexpr uint32_t kProbeRendezvousPolls = 1u << 16;  // both limits bound the wait at the start
 constexpr uint64_t kProbeRendezvousNs = 200000;       // 0.2 ms
+constexpr uint32_t kProbeExtraChunk = 64;             // reads between two looks at the other SM
 
 __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ ProbeArgs a)
 {
@@ -746,13 +631,40 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     uint64_t t_start = 0;
     if (threadIdx.x == 0) t_start = globaltimer();
     const uint64_t v = (uint64_t)sm * a.wps + warp;
+    const uint64_t key = sm64(a.key_seed ^ v), V = (uint64_t)a.nsm * a.wps;
+    const IndexSpec ix{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u, 0u, 0u};
     uint32_t X, S;
-    BulkRing no_ring{0u, 0u, 0u, nullptr, nullptr};
-    warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, sm64(a.key_seed ^ v),
-                                       IndexSpec{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u, 0u, 0u}, v,
-                                       (uint64_t)a.nsm * a.wps, 0, a.reads, 0u,
-                                       a.n_lines, lane, X, S, nullptr, no_ring);
-    if (lane == 0) a.out[which * a.wps + warp] = make_uint2(X, S);
+    WarpScratch no_ring{nullptr};
+    warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, key, ix, v, V, 0, a.reads, 0u,
+                                         a.n_lines, lane, X, S, nullptr, no_ring);
+    if (lane == 0) {
+        a.out[which * a.wps + warp] = make_uint2(X, S);
+        atomicAdd(&a.rec->done_warps[which], 1u);
+    }
+    // The fixed share is done (and is what the checksums cover).  Two SMs rarely finish together
+    // -- solo rates differ by +-12 % between SMs -- and a tail in which one SM runs alone would
+    // read as less contention.  So the warp keeps reading its stream, a short chunk at a time,
+    // until every warp of the other SM has finished its share; the host counts these lines too.
+    // Bounded: at most as many lines again as the share itself.
+    if (a.sm_b != 0xFFFFFFFFu) {
+        uint64_t extra = 0;
+        uint32_t keep = 0;
+        while (extra < a.reads) {
+            uint32_t d = 0;
+            if (lane == 0) d = *reinterpret_cast<volatile uint32_t *>(&a.rec->done_warps[which ^ 1u]);
+            if (__shfl_sync(0xFFFFFFFFu, d, 0) >= a.wps) break;
+            uint32_t x2, s2;
+            warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, key, ix, v, V,
+                                                 a.reads + extra, kProbeExtraChunk, 0u, a.n_lines,
+                                                 lane, x2, s2, nullptr, no_ring);
+            keep ^= x2 + s2;
+            extra += kProbeExtraChunk;
+        }
+        if (lane == 0 && extra) {
+            atomicAdd(&a.rec->extra_lines[which], (unsigned long long)extra);
+            atomicXor(&a.rec->sink, keep);
+        }
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         a.rec->t_start[which] = t_start;
@@ -789,19 +701,6 @@ static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
             default: return read_kernel<2, 2, kVarSorted>;
         }
     }
-    if (variant == RR_VARIANT_L2_128 || variant == RR_VARIANT_L2_256 ||
-        variant == RR_VARIANT_BULK) {  // comparison variants: ring depth 4 or 8 only
-#define RR_CMP_ROW(W_)                                                                  \
-    if (W == W_) {                                                                      \
-        if (variant == RR_VARIANT_L2_128) return read_kernel<W_, 8, kVarL2_128>;        \
-        if (variant == RR_VARIANT_L2_256) return read_kernel<W_, 8, kVarL2_256>;        \
-        return U == 4 ? read_kernel<W_, 4, kVarBulk> : read_kernel<W_, 8, kVarBulk>;    \
-    }
-        RR_CMP_ROW(1)
-        RR_CMP_ROW(2)
-        RR_CMP_ROW(4)
-#undef RR_CMP_ROW
-    }
     const bool checked = variant == RR_VARIANT_LDG_CHECKED;
 #define RR_ROW(W_, UMAX_)                                                               \
     if (W == W_) {                                                                      \
@@ -818,13 +717,6 @@ static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
     RR_ROW(4, 8)
 #undef RR_ROW
     return nullptr;
-}
-
-// Shared memory the bulk shape needs: per warp a ring of U lines and U mbarriers.
-static size_t bulk_smem_bytes(uint32_t variant, uint32_t W, uint32_t U, uint32_t warps_per_block)
-{
-    if (variant != RR_VARIANT_BULK) return 0;
-    return (size_t)warps_per_block * U * (128u * W + 8u);
 }
 
 static bool width_ok(uint32_t W) { return W == 1 || W == 2 || W == 4; }
@@ -868,9 +760,6 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_SORTED ? 2u : packed_shape ? 4u : 8u);
     if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && packed_shape)) return RR_ERR_ARG;
     if (p->variant == RR_VARIANT_SORTED && U > 4) return RR_ERR_ARG;
-    if ((p->variant == RR_VARIANT_L2_128 || p->variant == RR_VARIANT_L2_256) && U != 8)
-        return RR_ERR_ARG;
-    if (p->variant == RR_VARIANT_BULK && U != 4 && U != 8) return RR_ERR_ARG;
     if (U * p->words_per_lane > 32) U = 32 / p->words_per_lane;  // the ring holds 32 words a lane
     *unroll = U;
     if ((uintptr_t)p->buf % 512u) return RR_ERR_ALIGN;
@@ -951,19 +840,16 @@ static int32_t geometry(const rr_read_params_t *p, const DeviceFacts &f, Geometr
 
 // ---- launch configuration, found once per (device, kernel, block size, blocks per SM) -----------
 // Smallest dynamic shared-memory request that makes exactly `want` blocks of `block` threads
-// resident per SM (so that a grid of nsm*want blocks puts `want` on every SM), raised to `need`
-// when the kernel really uses dynamic shared memory.  The occupancy search costs ~100 runtime
-// calls, so its result is kept for the life of the process; later launches of the same
-// configuration make no occupancy or attribute call at all.
+// resident per SM, so that a grid of nsm*want blocks puts `want` on every SM.  The occupancy
+// search costs ~100 runtime calls, so its result is kept for the life of the process; later
+// launches of the same configuration make no occupancy or attribute call at all.
 struct LaunchKey {
     int device;
     const void *kernel;
     int block, want;
-    size_t need;
     bool operator==(const LaunchKey &o) const
     {
-        return device == o.device && kernel == o.kernel && block == o.block && want == o.want &&
-               need == o.need;
+        return device == o.device && kernel == o.kernel && block == o.block && want == o.want;
     }
 };
 struct LaunchEntry {
@@ -974,27 +860,19 @@ static std::mutex g_launch_mutex;
 static std::vector<LaunchEntry> g_launch_cache;
 static std::atomic<uint64_t> g_n_occupancy_queries{0}, g_n_attribute_sets{0}, g_n_event_creates{0};
 
-static int32_t search_ballast(const void *kernel, int block, int want, size_t need,
-                              const DeviceFacts &f, size_t *smem_out)
+static int32_t search_ballast(const void *kernel, int block, int want, const DeviceFacts &f,
+                              size_t *smem_out)
 {
     cudaFuncAttributes fa;
     RR_CUDA(cudaFuncGetAttributes(&fa, kernel));
     const int per_block_reserved = 1024;
     const int stat = (int)fa.sharedSizeBytes;
     const int most = f.smem_per_block_optin - stat;  // the largest request one block may make
-    if ((int)need > most) {
-        set_cuda_error(cudaErrorLaunchOutOfResources, "shared-memory ring does not fit");
-        return RR_ERR_CUDA;
-    }
     // one opt-in to the largest request any configuration of this kernel may make; the attribute
     // is a permission, it does not change residency
     g_n_attribute_sets.fetch_add(1);
     RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  std::max(most, 0)));
-    if (want <= 0) {  // no residency requirement (LOGICAL mode): just the ring
-        *smem_out = need;
-        return RR_OK;
-    }
     auto blocks_at = [&](size_t smem, int *nb) -> int32_t {
         g_n_occupancy_queries.fetch_add(1);
         RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, kernel, block, smem));
@@ -1003,7 +881,7 @@ static int32_t search_ballast(const void *kernel, int block, int want, size_t ne
     int lo = f.smem_per_sm / (want + 1) - per_block_reserved - stat + 1;
     if (lo < 0) lo = 0;
     const int hi = std::min(most, f.smem_per_sm / want - per_block_reserved - stat);
-    for (int smem = std::max(lo, (int)need); smem <= hi; smem += 1024) {
+    for (int smem = lo; smem <= hi; smem += 1024) {
         int nb = 0;
         int32_t rc = blocks_at((size_t)smem, &nb);
         if (rc != RR_OK) return rc;
@@ -1015,10 +893,10 @@ static int32_t search_ballast(const void *kernel, int block, int want, size_t ne
     }
     // registers or threads already limit residency below `want`
     int nb = 0;
-    int32_t rc = blocks_at(need, &nb);
+    int32_t rc = blocks_at(0, &nb);
     if (rc != RR_OK) return rc;
     if (nb == want) {
-        *smem_out = need;
+        *smem_out = 0;
         return RR_OK;
     }
     set_cuda_error(cudaErrorLaunchOutOfResources, "cannot force the requested blocks per SM");
@@ -1026,10 +904,10 @@ static int32_t search_ballast(const void *kernel, int block, int want, size_t ne
 }
 
 template <typename K>
-static int32_t launch_smem(K kernel, int block, int want, size_t need, const DeviceFacts &f,
-                           size_t *smem_out)
+static int32_t launch_smem(K kernel, int block, int want, const DeviceFacts &f, size_t *smem_out)
 {
-    const LaunchKey key{f.device, (const void *)kernel, block, want, need};
+    if (want <= 0) return RR_ERR_ARG;
+    const LaunchKey key{f.device, (const void *)kernel, block, want};
     std::lock_guard<std::mutex> lock(g_launch_mutex);
     for (const LaunchEntry &e : g_launch_cache)
         if (e.key == key) {
@@ -1037,7 +915,7 @@ static int32_t launch_smem(K kernel, int block, int want, size_t need, const Dev
             return RR_OK;
         }
     size_t smem = 0;
-    int32_t rc = search_ballast((const void *)kernel, block, want, need, f, &smem);
+    int32_t rc = search_ballast((const void *)kernel, block, want, f, &smem);
     if (rc != RR_OK) return rc;
     g_launch_cache.push_back(LaunchEntry{key, smem});
     *smem_out = smem;
@@ -1142,7 +1020,6 @@ static int32_t decode(const rr_read_params_t *p, const Geometry &g, const Device
     res->violations = h.violations;
     res->sms_covered = covered;
     res->blocks_run = h.blocks_run;
-    if (h.status & kStatusBulkTimeout) return RR_ERR_TIMEOUT;
     if (uncovered) return RR_ERR_SM_UNCOVERED;
     if (h.violations) return RR_ERR_CHECK;
     if (h.status) return RR_ERR_SM_UNCOVERED;
@@ -1170,10 +1047,8 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     cudaStream_t stream = (cudaStream_t)stream_;
 
     size_t smem = 0;
-    const size_t need = bulk_smem_bytes(p->variant, p->words_per_lane, U, g.wpc);
-    if (p->mode != RR_MODE_LOGICAL || need) {
-        rc = launch_smem(kernel, (int)g.block, p->mode != RR_MODE_LOGICAL ? (int)g.cps : 0, need, f,
-                         &smem);
+    if (p->mode != RR_MODE_LOGICAL) {
+        rc = launch_smem(kernel, (int)g.block, (int)g.cps, f, &smem);
         if (rc != RR_OK) return rc;
     }
 
@@ -1295,31 +1170,34 @@ static ProbeArgs probe_args(const void *buf, uint64_t region_bytes, uint32_t a, 
 static bool probe_rate(const ProbeRecord &r, bool solo, uint64_t total_reads, double *gbps,
                        double *seconds, double *overlap)
 {
-    return rr_probe_rate(r.t_start, r.t_end, r.claim, solo ? 1u : 0u, total_reads, gbps, seconds,
-                         overlap) == RR_OK;
+    const uint64_t extra[2] = {r.extra_lines[0], r.extra_lines[1]};
+    return rr_probe_rate(r.t_start, r.t_end, r.claim, extra, solo ? 1u : 0u, total_reads, gbps,
+                         seconds, overlap) == RR_OK;
 }
 
 }  // namespace rr
 
 // Bytes of both SMs over the union of their intervals; overlap = intersection / union.
 extern "C" int32_t rr_probe_rate(const uint64_t *t_start, const uint64_t *t_end,
-                                 const uint32_t *claim, uint32_t solo, uint64_t total_reads,
-                                 double *gbps, double *seconds, double *overlap)
+                                 const uint32_t *claim, const uint64_t *extra_lines, uint32_t solo,
+                                 uint64_t total_reads, double *gbps, double *seconds,
+                                 double *overlap)
 {
-    if (!t_start || !t_end || !claim || !gbps || !seconds || !overlap || solo > 1) return RR_ERR_ARG;
+    if (!t_start || !t_end || !claim || !extra_lines || !gbps || !seconds || !overlap || solo > 1)
+        return RR_ERR_ARG;
     const int k = solo ? 1 : 2;
-    uint64_t first_start = ~0ull, last_start = 0, first_end = ~0ull, last_end = 0;
+    uint64_t first_start = ~0ull, last_start = 0, first_end = ~0ull, last_end = 0, lines = 0;
     for (int i = 0; i < k; ++i) {
         if (claim[i] == 0 || t_end[i] == 0 || t_end[i] < t_start[i]) return RR_ERR_SM_UNCOVERED;
         first_start = std::min(first_start, t_start[i]);
         last_start = std::max(last_start, t_start[i]);
         first_end = std::min(first_end, t_end[i]);
         last_end = std::max(last_end, t_end[i]);
+        lines += total_reads / 2 + extra_lines[i];
     }
     const uint64_t uni = last_end - first_start;
-    const uint64_t bytes = (total_reads / 2) * (uint64_t)k * 128ull;
     *seconds = (double)uni * 1e-9;
-    *gbps = uni ? (double)bytes / (double)uni : 0.0;  // bytes per ns = GB/s
+    *gbps = uni ? (double)(lines * 128ull) / (double)uni : 0.0;  // bytes per ns = GB/s
     *overlap = (uni && first_end > last_start) ? (double)(first_end - last_start) / (double)uni : 0.0;
     return RR_OK;
 }
@@ -1337,6 +1215,7 @@ namespace rr {
 
 struct ProbeSample {
     double gbps, seconds, overlap, seconds_event;
+    uint64_t extra_lines;
 };
 
 // One probe launch on its own (synchronous), retried with larger grids if a chosen SM got no
@@ -1365,6 +1244,7 @@ static int32_t probe_once(const void *buf, uint64_t region_bytes, uint32_t sm_a,
         RR_CUDA(cudaEventElapsedTime(&ms, ev->e0, ev->e1));
         if (probe_rate(h, sm_a == sm_b, total_reads, &out->gbps, &out->seconds, &out->overlap)) {
             out->seconds_event = (double)ms * 1e-3;
+            out->extra_lines = h.extra_lines[0] + h.extra_lines[1];
             return RR_OK;
         }
     }
@@ -1385,7 +1265,7 @@ extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_
     if (rc != RR_OK) return rc;
     if (sm_a >= (uint32_t)f.nsm || sm_b >= (uint32_t)f.nsm) return RR_ERR_ARG;
     size_t smem = 0;
-    rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
+    rc = launch_smem(probe_kernel, (int)wps * 32, 1, f, &smem);
     if (rc != RR_OK) return rc;
     std::memset(res, 0, sizeof(*res));
     ProbeSample s;
@@ -1394,7 +1274,7 @@ extern "C" int32_t rr_probe_pair(const void *buf, uint64_t region_bytes, uint32_
     if (rc != RR_OK) return rc;
     res->seconds_event = s.seconds_event;
     res->seconds_device = s.seconds;
-    res->bytes = (total_reads / 2) * (sm_a == sm_b ? 1 : 2) * 128ull;
+    res->bytes = ((total_reads / 2) * (sm_a == sm_b ? 1 : 2) + s.extra_lines) * 128ull;
     res->gbps = s.gbps;
     res->sms_covered = sm_a == sm_b ? 1 : 2;
     res->blocks_run = res->sms_covered;
@@ -1423,7 +1303,7 @@ extern "C" int32_t rr_probe_rows(const void *buf, uint64_t region_bytes, uint64_
     if (nsm != (uint32_t)f.nsm) return RR_ERR_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    rc = launch_smem(probe_kernel, (int)wps * 32, 1, 0, f, &smem);
+    rc = launch_smem(probe_kernel, (int)wps * 32, 1, f, &smem);
     if (rc != RR_OK) return rc;
 
     size_t n_pairs = 0;  // pairs (a, b >= a) of the requested rows
@@ -1461,7 +1341,7 @@ extern "C" int32_t rr_probe_rows(const void *buf, uint64_t region_bytes, uint64_
         k = 0;
         for (uint32_t a = row_begin; a < row_end; ++a)
             for (uint32_t b = a; b < nsm; ++b, ++k) {
-                ProbeSample best{0, 0, 0, 0};
+                ProbeSample best{0, 0, 0, 0, 0};
                 bool have = probe_rate(h[k], a == b, total_reads, &best.gbps, &best.seconds,
                                        &best.overlap);
                 if (!have) {
@@ -1579,9 +1459,8 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     if (rc != RR_OK) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    const size_t need = bulk_smem_bytes(p->variant, p->words_per_lane, U, g.wpc);
-    if (p->mode == RR_MODE_PER_SM || need) {
-        rc = launch_smem(kernel, (int)g.block, p->mode == RR_MODE_PER_SM ? 1 : 0, need, f, &smem);
+    if (p->mode == RR_MODE_PER_SM) {
+        rc = launch_smem(kernel, (int)g.block, 1, f, &smem);
         if (rc != RR_OK) return rc;
     }
     ReadArgs a;

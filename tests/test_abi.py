@@ -323,14 +323,15 @@ def test_probe_rate_matches_oracle():
             t1[int(rng.integers(0, 2))] = 0
         solo = bool(rng.random() < 0.3)
         reads = int(rng.integers(1, 1 << 24)) * 2
+        extra = rng.integers(0, 1 << 20, 2).astype(np.uint64) * 64
         try:
-            expect = oracle.probe_rate(t0, t1, claim, solo, reads)
+            expect = oracle.probe_rate(t0, t1, claim, solo, reads, extra)
         except oracle.OracleError as e:
             with pytest.raises(rr.RRError) as r:
-                rr.rr_probe_rate(t0, t1, claim, solo, reads)
+                rr.rr_probe_rate(t0, t1, claim, solo, reads, extra)
             assert r.value.code == e.code == rr.RR_ERR_SM_UNCOVERED
             continue
-        assert rr.rr_probe_rate(t0, t1, claim, solo, reads) == expect
+        assert rr.rr_probe_rate(t0, t1, claim, solo, reads, extra) == expect
 
 
 def test_exact_remainder_identity():

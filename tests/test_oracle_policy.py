@@ -287,6 +287,9 @@ def test_probe_rate_hand_worked():
     # solo: one SM's bytes, overlap 1 by definition, the second entry is ignored
     g, sec, ov = oracle.probe_rate([100, 0], [1100, 0], [1, 0], True, reads)
     assert (g, ov) == (262144 / 1000, 1.0)
+    # lines read beyond the fixed share (an SM that waited for a slower partner) count as well
+    g, sec, ov = oracle.probe_rate([100, 100], [1100, 1090], [1, 1], False, reads, extra_lines=(0, 192))
+    assert g == (524288 + 192 * 128) / 1000 and ov == 990 / 1000
     # an SM that never ran
     for bad in ([[100, 100], [1100, 0], [1, 1]], [[100, 100], [1100, 1100], [1, 0]]):
         with pytest.raises(oracle.OracleError) as e:
