@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--region-bytes B]
 
-Metric (the benchmark spec): random 128-B line read GB/s over the full HBM with SM groups held to
+Metric: random 128-B line read GB/s over the full HBM with SM groups held to
 address windows below the measured translation reach, next to the unrestricted rate.
 
 One step = one launch of the persistent read kernel over ~95 % of free HBM: 148 x 32 logical
@@ -59,6 +59,7 @@ SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
 NSM_NOMINAL = 148
+RR_MAX_SM_FOR_SCRATCH = 192   # the sorted arm's index scratch is sized before the SM count is known
 # DRAM bytes moved per algorithmic byte by the read kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over lines x 128 B, 4 GiB case).
 TRAFFIC_PER_ALGORITHMIC_BYTE = 0.975
@@ -164,7 +165,8 @@ def run_gpu(args):
     from paper_2405_11425_b200 import binding as rr
     from paper_2405_11425_b200 import build as rr_build
     from paper_2405_11425_b200.clocks import ClockSampler
-    from paper_2405_11425_b200.pipeline import Session, aggregate_throughput
+    from paper_2405_11425_b200.pipeline import (Session, aggregate_throughput, load_calibration,
+                                                 save_calibration)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -187,15 +189,29 @@ def run_gpu(args):
 
     # ---- calibration (untimed): fill, groups, reach ---------------------------------------------
     t_cal = time.time()
+    sort_scratch = torch.empty(rr.rr_sort_scratch_bytes(RR_MAX_SM_FOR_SCRATCH, 4, 1024),
+                               dtype=torch.uint8, device="cuda")   # before the region takes the rest
     ses = Session()
     N = ses.region_bytes
     fill_gbps = max(ses.fill(), ses.fill())
-    groups = ses.discover_groups(total_reads=args.probe_reads, repeats=args.probe_repeats)
+    loaded = None
+    if args.load_calibration:
+        # the layout is a property of the card: a calibration saved on this very GPU is reused
+        loaded = load_calibration(args.load_calibration, ses.info["uuid"], ses.nsm, with_extra=True)
+        if loaded[3].get("region_bytes") != N:
+            raise SystemExit("bench.py: the saved calibration was taken with another buffer size")
+    if loaded:
+        groups, reach, grp_weights_saved, saved = loaded
+        sm_reach = int(saved["sm_reach_bytes"])
+        sm_reach_points = [tuple(x) for x in saved["sm_reach_points"]]
+        t_reach = 0.0
+    else:
+        groups = ses.discover_groups(total_reads=args.probe_reads, repeats=args.probe_repeats)
+        t_reach = time.time()
+        reach = ses.measure_reach(variant=VARIANT_PACKED, unroll=UNROLL)
+        t_reach = time.time() - t_reach
+        sm_reach, sm_reach_points = ses.measure_sm_reach()
     gpc, n_gpc = rr.rr_gpc_map(ses.scratch, ses.nsm)
-    t_reach = time.time()
-    reach = ses.measure_reach(variant=VARIANT_PACKED, unroll=UNROLL)
-    t_reach = time.time() - t_reach
-    sm_reach, sm_reach_points = ses.measure_sm_reach()
     t_cal = time.time() - t_cal
 
     # ---- the arms of the comparison, all by one protocol ------------------------------------------
@@ -227,35 +243,36 @@ def run_gpu(args):
     arms["b_unrestricted_inside_one_window"] = measure(
         ses.params(S, W=1, seed=SEED, reads_per_warp=arm_reads, **kern),
         window_gib_min_max=[S / GiB, S / GiB], coverage=S / N)
+    full = args.arms == "all"
     cfg4 = {}
     for name, S_w in sweep_sizes.items():
+        if not full and name != headline:
+            continue
         win, cov = ses.windows(groups, S_w)
         cfg4[name] = measure(ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads,
                                         group_of_sm=groups.group_of_sm, windows=win, **kern),
                              win, coverage=cov, window_gib_asked=S_w / GiB)
     arms["c_one_window_per_group_equal_work_per_sm"] = cfg4
-    win256, cov256 = ses.windows(groups, S, W=2)
-    arms["c_256B_lines_one_window_per_group"] = measure(
-        ses.params(N, W=2, seed=SEED, reads_per_warp=arm_reads, group_of_sm=groups.group_of_sm,
-                   windows=win256, **kern), win256, coverage=cov256)
-    arms["a_256B_lines_unrestricted_whole_buffer"] = measure(
-        ses.params(N, W=2, seed=SEED, reads_per_warp=arm_reads, **kern), coverage=1.0)
-    ctrl_groups, ctrl_win, ctrl_cov = ses.naive_control(S, SEED)
-    arms["c3_naive_per_sm_control"] = measure(
-        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=ctrl_groups,
-                   windows=ctrl_win, **kern), ctrl_win, coverage=ctrl_cov)
-    ov_win, ov_cov = rr.rr_make_windows(N, 1, S, groups.n_groups, policy=2)
-    covered, dmin, dmax = rr.rr_window_cover(ov_win, N // 128)
-    arms["c_overlapping_windows_per_group"] = measure(
-        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=groups.group_of_sm,
-                   windows=ov_win, **kern), ov_win, coverage=ov_cov, depth_min_max=[dmin, dmax])
+    if full:
+        win256, cov256 = ses.windows(groups, S, W=2)
+        arms["c_256B_lines_one_window_per_group"] = measure(
+            ses.params(N, W=2, seed=SEED, reads_per_warp=arm_reads, group_of_sm=groups.group_of_sm,
+                       windows=win256, **kern), win256, coverage=cov256)
+        arms["a_256B_lines_unrestricted_whole_buffer"] = measure(
+            ses.params(N, W=2, seed=SEED, reads_per_warp=arm_reads, **kern), coverage=1.0)
+        ctrl_groups, ctrl_win, ctrl_cov = ses.naive_control(S, SEED)
+        arms["c3_naive_per_sm_control"] = measure(
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=ctrl_groups,
+                       windows=ctrl_win, **kern), ctrl_win, coverage=ctrl_cov)
+        ov_win, ov_cov = rr.rr_make_windows(N, 1, S, groups.n_groups, policy=2)
+        covered, dmin, dmax = rr.rr_window_cover(ov_win, N // 128)
+        arms["c_overlapping_windows_per_group"] = measure(
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=groups.group_of_sm,
+                       windows=ov_win, **kern), ov_win, coverage=ov_cov, depth_min_max=[dmin, dmax])
 
     # work and window size in proportion to capacity with everything running (pooled mode)
     max_window = reach.reach_bytes if reach.cliff else 0
     t_bal = time.time()
-    grp_win, grp_ws, grp_weights, grp_hist = ses.balance(
-        groups, W=1, n_warps=n_warps, reads_per_warp=arm_reads, seed=SEED,
-        max_window_bytes=max_window, launches_per_round=100, rounds=8, **kern)
 
     def pooled(owner_map, windows, warp_start, reads, first_read=0):
         return ses.params(N, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
@@ -263,40 +280,60 @@ def run_gpu(args):
                           seed=SEED, group_of_sm=owner_map, windows=windows, warp_start=warp_start,
                           **kern)
 
-    arms["d_pooled_one_window_per_group"] = measure(
-        pooled(groups.group_of_sm, grp_win, grp_ws, arm_reads), grp_win, coverage=1.0,
-        gbps_by_balancing_round=grp_hist)
     # one window per SM, side by side inside the SM's resource group (rr_owner_map)
     owners = ses.singleton_groups(groups)
-    bal_windows, warp_start, weights, bal_history = ses.balance(
-        owners, W=1, n_warps=n_warps, reads_per_warp=arm_reads, seed=SEED,
-        max_window_bytes=max_window, launches_per_round=150, rounds=8, **kern)
+    if loaded:
+        grp_weights = grp_weights_saved
+        weights = np.asarray(saved["weights_per_window"], dtype=np.uint32)
+        grp_win, grp_ws = rr.rr_make_weighted_windows(N, 1, grp_weights, n_warps, max_window)
+        bal_windows, warp_start = rr.rr_make_weighted_windows(N, 1, weights, n_warps, max_window)
+        grp_hist = bal_history = []
+    else:
+        grp_win, grp_ws, grp_weights, grp_hist = ses.balance(
+            groups, W=1, n_warps=n_warps, reads_per_warp=arm_reads, seed=SEED,
+            max_window_bytes=max_window, launches_per_round=100, rounds=8, **kern)
+        bal_windows, warp_start, weights, bal_history = ses.balance(
+            owners, W=1, n_warps=n_warps, reads_per_warp=arm_reads, seed=SEED,
+            max_window_bytes=max_window, launches_per_round=150, rounds=8, **kern)
     t_bal = time.time() - t_bal
+    if args.save_calibration and rank == 0:
+        save_calibration(args.save_calibration, ses.info["uuid"], groups, reach, grp_weights,
+                         extra={"region_bytes": N, "sm_reach_bytes": int(sm_reach),
+                                "sm_reach_points": [[int(b), float(g)] for b, g in sm_reach_points],
+                                "weights_per_window": [int(w) for w in weights]})
+    if full:
+        arms["d_pooled_one_window_per_group"] = measure(
+            pooled(groups.group_of_sm, grp_win, grp_ws, arm_reads), grp_win, coverage=1.0,
+            gbps_by_balancing_round=grp_hist)
     arms["e_pooled_one_window_per_sm"] = measure(
         pooled(owners.group_of_sm, bal_windows, warp_start, arm_reads), bal_windows, coverage=1.0,
         gbps_by_balancing_round=bal_history)
 
-    # moving windows: the same per-SM slices (equal size, equal work), read one sub-window at a time
-    mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
-    slice_bytes = int(mv_windows[:, 1].max()) * 128
-    mv_parts, mv_sub = rr.rr_phase_window(slice_bytes, sm_reach, 64)
-    phased = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=1024, phase_window_bytes=mv_sub)
-    arms["f_moving_sub_windows_per_sm_slices"] = measure(
-        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
-                   windows=mv_windows, **kern, **phased), mv_windows, coverage=1.0,
-        sub_window_mib=mv_sub / (1 << 20), sub_windows=mv_parts, phase_reads=1024)
-    arms["f_moving_sub_windows_no_partition"] = measure(
-        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, **kern, **phased),
-        window_gib_min_max=[N / GiB, N / GiB], coverage=1.0,
-        sub_window_mib=mv_sub / (1 << 20), phase_reads=1024,
-        note="every SM's window is the whole buffer; SM cycles staggered")
-    # static per-SM slices, equal work, no calibration of weights: the kernel performs each warp's
-    # reads part by part of its window (same reads and checksums, another order)
-    arms["g_sorted_execution_static_per_sm_slices"] = measure(
-        ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
-                   windows=mv_windows, variant=VARIANT_SORTED, unroll=1, sort_parts=4,
-                   sort_reads=1024), mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
-        kernel="read_kernel<U=1, sorted>")
+    if full:
+        # moving windows: the same per-SM slices (equal size, equal work), one sub-window at a time
+        mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
+        slice_bytes = int(mv_windows[:, 1].max()) * 128
+        mv_parts, mv_sub = rr.rr_phase_window(slice_bytes, sm_reach, 64)
+        phased = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=1024, phase_window_bytes=mv_sub)
+        arms["f_moving_sub_windows_per_sm_slices"] = measure(
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
+                       windows=mv_windows, **kern, **phased), mv_windows, coverage=1.0,
+            sub_window_mib=mv_sub / (1 << 20), sub_windows=mv_parts, phase_reads=1024)
+        arms["f_moving_sub_windows_no_partition"] = measure(
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, **kern, **phased),
+            window_gib_min_max=[N / GiB, N / GiB], coverage=1.0,
+            sub_window_mib=mv_sub / (1 << 20), phase_reads=1024,
+            note="every SM's window is the whole buffer; SM cycles staggered")
+        # static per-SM slices, equal work, no calibration of weights: the kernel performs each
+        # warp's reads part by part of its window (same reads and checksums, another order)
+        for cached in (False, True):
+            arms["g_sorted_execution_static_per_sm_slices" + ("_cached" if cached else "")] = measure(
+                ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads,
+                           group_of_sm=owners.group_of_sm, windows=mv_windows,
+                           variant=VARIANT_SORTED, unroll=1, sort_parts=4, sort_reads=1024,
+                           sort_scratch=sort_scratch if cached else None),
+                mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
+                kernel="read_kernel<U=1, sorted>" + (", indices cached" if cached else ""))
     t_arms = time.time() - t_arms
     c_head = cfg4[headline]["gbps"]
     comparison = {
@@ -437,9 +474,10 @@ def run_gpu(args):
                             "in proportion to measured capacity (pooled mode), seed 23; the "
                             "paper's one-window-per-group policy is arms.c / arms.d",
                 "one_window_per_group_gbps": {"equal_work_per_sm": c_head,
-                                              "capacity_weighted": arms[
-                                                  "d_pooled_one_window_per_group"]["gbps"],
+                                              "capacity_weighted": arms.get(
+                                                  "d_pooled_one_window_per_group", {}).get("gbps"),
                                               "window_gib": S / GiB},
+                "arms_measured": args.arms,
                 "region_bytes": N, "region_gib": N / GiB, "line_bytes": 128,
                 "logical_warps": n_warps, "warps_per_sm": WARPS_PER_SM,
                 "reads_per_warp_per_step": reads,
@@ -471,6 +509,7 @@ def run_gpu(args):
             "calibration": {
                 "device": ses.info["name"], "uuid": ses.info["uuid"], "nsm": ses.nsm,
                 "seconds_total": t_cal, "seconds_reach_sweep": t_reach,
+                "loaded_from_file": bool(loaded),
                 "fill_gbps": fill_gbps,
                 "probe": {"seconds": groups.probe_seconds, "pairs": ses.nsm * (ses.nsm + 1) // 2,
                           "reads_per_pair": args.probe_reads, "repeats": args.probe_repeats,
@@ -508,6 +547,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--probe-reads", type=int, default=1 << 18)
     ap.add_argument("--probe-repeats", type=int, default=3)
+    ap.add_argument("--arms", default="all", choices=["all", "headline"],
+                    help="headline: only the arms value and comparison need (a, b, c at the "
+                         "headline window, e)")
+    ap.add_argument("--save-calibration", default="",
+                    help="write groups, reach and weights of this card to a JSON file")
+    ap.add_argument("--load-calibration", default="",
+                    help="reuse a file written by --save-calibration on this very GPU instead "
+                         "of probing, sweeping and balancing again")
     ap.add_argument("--region-bytes", type=int, default=0,
                     help="reference arm: region size (default: 0.95 of free HBM if a GPU is "
                          "visible, else a nominal B200)")

@@ -60,23 +60,27 @@ def aggregate_throughput(local_bytes: float, local_seconds: float, group=None) -
 
 
 def save_calibration(path, uuid: str, groups: "Groups", reach: "Reach | None" = None,
-                     weights=None) -> None:
-    """Writes what was measured on one card (SM groups, reach, capacity weights) as JSON, keyed by
-    the GPU's UUID: the layout is a property of the card (Section 1.1), so it can be reused."""
+                     weights=None, extra: dict | None = None) -> None:
+    """Writes what was measured on one card (SM groups, reach, capacity weights, and whatever
+    else the caller adds under `extra`) as JSON, keyed by the GPU's UUID: the layout is a
+    property of the card (Section 1.1), so it can be reused."""
     import json
     doc = {"uuid": uuid, "n_groups": int(groups.n_groups), "confidence": float(groups.confidence),
            "group_of_sm": [int(g) for g in groups.group_of_sm],
+           "probe_stats": groups.probe_stats, "probe_seconds": float(groups.probe_seconds),
            "reach": None if reach is None else {"cliff": bool(reach.cliff),
                                                 "plateau_gbps": float(reach.plateau_gbps),
-                                                "reach_bytes": int(reach.reach_bytes)},
-           "weights": None if weights is None else [int(w) for w in weights]}
+                                                "reach_bytes": int(reach.reach_bytes),
+                                                "sweep": [[int(s), float(g)] for s, g in reach.sweep]},
+           "weights": None if weights is None else [int(w) for w in weights],
+           "extra": extra or {}}
     with open(path, "w") as f:
         json.dump(doc, f)
 
 
-def load_calibration(path, uuid: str, nsm: int):
+def load_calibration(path, uuid: str, nsm: int, with_extra: bool = False):
     """Reads a calibration written by save_calibration; refuses one taken on another card or with
-    another SM count.  Returns (Groups, Reach or None, weights or None)."""
+    another SM count.  Returns (Groups, Reach or None, weights or None[, extra])."""
     import json
     with open(path) as f:
         doc = json.load(f)
@@ -85,13 +89,17 @@ def load_calibration(path, uuid: str, nsm: int):
     g = np.asarray(doc["group_of_sm"], dtype=np.uint16)
     if g.shape != (nsm,) or int(g.max()) + 1 != doc["n_groups"]:
         raise ValueError("calibration does not describe this SM count")
-    groups = Groups(g, int(doc["n_groups"]), float(doc["confidence"]), None, 1.0, 0.0,
-                    np.bincount(g, minlength=doc["n_groups"]).tolist())
+    stats = doc.get("probe_stats") or {}
+    groups = Groups(g, int(doc["n_groups"]), float(doc["confidence"]), None,
+                    float(stats.get("overlap_min", 1.0)), float(doc.get("probe_seconds", 0.0)),
+                    np.bincount(g, minlength=doc["n_groups"]).tolist(), stats)
     r = doc.get("reach")
     reach = None if r is None else Reach(bool(r["cliff"]), float(r["plateau_gbps"]),
-                                         int(r["reach_bytes"]), [])
+                                         int(r["reach_bytes"]),
+                                         [(int(s), float(x)) for s, x in r.get("sweep", [])])
     w = doc.get("weights")
-    return groups, reach, None if w is None else np.asarray(w, dtype=np.uint32)
+    out = (groups, reach, None if w is None else np.asarray(w, dtype=np.uint32))
+    return out + (doc.get("extra") or {},) if with_extra else out
 
 
 class Session:

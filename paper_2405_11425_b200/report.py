@@ -2,7 +2,7 @@
 
     python -m paper_2405_11425_b200.report --out DIR [--quick]
 
-Experiments (paper section -> BASELINE config):
+Experiments (paper section -> workload configuration):
   size sweep, unrestricted            Section 2.1, Fig. 1            configs[1]
   line widths at 32 GiB               Section 2.1                    configs[2]
   pair probe + clustering             Section 2.2, Fig. 2-3          configs[3]
@@ -10,8 +10,9 @@ Experiments (paper section -> BASELINE config):
   grouped windows over all memory     Section 2.4, Fig. 6            configs[4]
   sequential reads of the same kernel Section 2.1 (last paragraph)
   allocation paths (--alloc-study)    Section 1.2 (reach = translations x page size)
-All numbers are event-timed GB/s (10^9 B/s), median of the repetitions; nothing is computed here
-beyond bookkeeping.
+All numbers are event-timed GB/s (10^9 B/s) by the sustained protocol of Session.sustained (settling
+launches, then regions of back-to-back launches; median [min-max] of the regions); nothing is
+computed here beyond bookkeeping.
 """
 from __future__ import annotations
 
@@ -26,11 +27,11 @@ from . import binding as rr
 from .pipeline import GiB, Session
 
 
-def _stats(ses, region, reps=5, **kw):
-    p = ses.params(region, **kw)
-    rr.rr_random_read(p, ses.out, ses.scratch)
-    r = sorted(rr.rr_random_read(p, ses.out, ses.scratch).gbps for _ in range(reps))
-    return {"median": r[(len(r) - 1) // 2], "min": r[0], "max": r[-1]}
+def _stats(ses, region, reps=5, *, settle=30, min_ms=50.0, **kw):
+    """One figure of the report: Session.sustained (settling launches, then `reps` regions of at
+    least `min_ms` of back-to-back launches), median / min / max GB/s."""
+    d = ses.sustained(ses.params(region, **kw), settle=settle, min_ms=min_ms, reps=reps)
+    return {"median": d["gbps"], "min": d["gbps_min"], "max": d["gbps_max"]}
 
 
 def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
@@ -75,6 +76,11 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     R["stride_full"] = {f"{128 * W}B": _stats(ses, N, reps, W=W, reads_per_warp=reads,
                                               index_mode=rr.RR_INDEX_STRIDE) for W in (1, 2, 4)}
 
+    # between the two: one read in k sequential, the rest random (32 GiB, inside the reach)
+    R["mixed_32gib"] = {str(k): _stats(ses, 32 * GiB, reps, W=1, seed=11, reads_per_warp=reads,
+                                       index_mode=rr.RR_INDEX_MIXED, mix_period=k)
+                        for k in (1, 2, 4, 16, 64)}
+
     # configs[3]: probe inside the reach (as the config says) and over everything
     t0 = time.time()
     g16 = ses.discover_groups(probe_region_bytes=16 * GiB,
@@ -107,8 +113,8 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     singles = []
     for g in range(groups.n_groups):
         gm = np.where(groups.group_of_sm == g, 0, 0xFFFF).astype(np.uint16)
-        rate = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=gm,
-                      windows=[[0, L_S]])["median"]
+        rate = _stats(ses, N, 3, settle=5, min_ms=20.0, seed=23, reads_per_warp=reads,
+                      group_of_sm=gm, windows=[[0, L_S]])["median"]
         singles.append({"group": g, "sms": int((gm == 0).sum()), "gbps": rate})
     R["single_groups"] = singles
     pairs = []
@@ -120,8 +126,8 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
         gm = np.full(ses.nsm, 0xFFFF, np.uint16)
         gm[groups.group_of_sm == a] = 0
         gm[groups.group_of_sm == b] = 1
-        rate = _stats(ses, N, 1, seed=23, reads_per_warp=reads, group_of_sm=gm,
-                      windows=[[0, L_S], [2 * L_S, L_S]])["median"]
+        rate = _stats(ses, N, 3, settle=5, min_ms=20.0, seed=23, reads_per_warp=reads,
+                      group_of_sm=gm, windows=[[0, L_S], [2 * L_S, L_S]])["median"]
         pairs.append({"a": a, "b": b, "gbps": rate,
                       "ratio_to_sum_of_singles": rate / (singles[a]["gbps"] + singles[b]["gbps"])})
     R["group_pairs_distinct_windows"] = pairs
@@ -217,6 +223,20 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
                                "sustained_gbps": rep.bytes * n / e0.elapsed_time(e1) * 1e-6})
     R["moving_windows_no_partition"] = moving_all
 
+    # sorted execution: the same static per-SM slices, equal work, each warp's reads taken part by
+    # part of its window -- hashing once per part, or once with the indices kept in a scratch
+    sorted_rows = []
+    for parts in (2, 4, 8):
+        cache = torch.empty(rr.rr_sort_scratch_bytes(ses.nsm, parts, 1024), dtype=torch.uint8,
+                            device="cuda")
+        for cached in (False, True):
+            d = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=owners_eq.group_of_sm,
+                       windows=eq_win, variant=rr.RR_VARIANT_SORTED, unroll=1, sort_parts=parts,
+                       sort_reads=1024, sort_scratch=cache if cached else None)
+            sorted_rows.append({"parts": parts, "cached": cached, **d})
+        del cache
+    R["sorted_execution"] = sorted_rows
+
     # work in proportion to group capacity (pooled mode), balanced under sustained load
     balanced = {}
     n_warps = ses.nsm * 32
@@ -291,6 +311,9 @@ def markdown(R: dict) -> str:
           "", "| line | random 32 GiB | sequential whole buffer |", "|---|---|---|"]
     for k in ("128B", "256B", "512B"):
         L.append(f"| {k} | {f(R['cfg2_widths_32gib'][k])} | {f(R['stride_full'][k])} |")
+    if "mixed_32gib" in R:
+        L += ["", "one read in k sequential, the others random (128-B lines, 32 GiB): "
+              + ", ".join(f"k={k}: {f(v)}" for k, v in R["mixed_32gib"].items())]
     p = R["cfg3_probe"]
     L += ["", "## Pair probe and clustering", "",
           f"inside the reach (16 GiB): {p['inside_reach_16gib']['n_groups']} group(s), pair GB/s "
@@ -338,6 +361,13 @@ def markdown(R: dict) -> str:
     for r in R.get("moving_windows_no_partition", []):
         L.append(f"| {r['sub_window_mib']} | {r['phase_reads']} | {r['sustained_gbps']:.0f} |")
     L.append("")
+    if "sorted_execution" in R:
+        L += ["## Sorted execution: static per-SM slices, equal work, reads taken part by part", "",
+              "| parts | indices | GB/s |", "|---|---|---|"]
+        for r in R["sorted_execution"]:
+            L.append(f"| {r['parts']} | {'hashed once, cached' if r['cached'] else 'hashed per part'} "
+                     f"| {f(r)} |")
+        L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]
     for name, b in R.get("balanced_pooled", {}).items():
