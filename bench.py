@@ -59,7 +59,6 @@ SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
 NSM_NOMINAL = 148
-RR_MAX_SM_FOR_SCRATCH = 192   # the sorted arm's index scratch is sized before the SM count is known
 # DRAM bytes moved per algorithmic byte by the read kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over lines x 128 B, 4 GiB case).
 TRAFFIC_PER_ALGORITHMIC_BYTE = 0.975
@@ -158,7 +157,33 @@ def _spawn_ranks(args):
     return subprocess.call(cmd)
 
 
+class NoSampler:
+    """Stands in for the clock sampler when it is switched off (--clock-period-ms 0), e.g. under a
+    profiler, where a concurrent nvidia-smi query loop slows every launch down."""
+
+    def wait_first_sample(self):
+        pass
+
+    def window(self, t_begin, t_end):
+        return {"sm_mhz": None, "sm_max_mhz": None, "power_w": None,
+                "reasons": ["sampler switched off"], "samples": 0, "during_timed_region": False}
+
+    def stop(self):
+        pass
+
+
 def run_gpu(args):
+    """Runs the benchmark; whatever happens, the nvidia-smi child of the clock sampler is stopped
+    (a profiler that follows child processes would otherwise wait for it for ever)."""
+    holder = {}
+    try:
+        return _run_gpu(args, holder)
+    finally:
+        if holder.get("sampler") is not None:
+            holder["sampler"].stop()
+
+
+def _run_gpu(args, holder):
     import torch
     import torch.distributed as dist
 
@@ -184,22 +209,26 @@ def run_gpu(args):
     if world > 1:
         dist.barrier()            # the other ranks load the library only after that
     peaks, peak_kind = _peaks()
-    sampler = ClockSampler(torch.cuda.current_device(), 50)
+    nvtx = torch.cuda.nvtx            # ranges let a profiler pick out the timed region
+    sampler = NoSampler() if args.clock_period_ms <= 0 else ClockSampler(
+        torch.cuda.current_device(), args.clock_period_ms)
+    holder["sampler"] = sampler
     sampler.wait_first_sample()
 
     # ---- calibration (untimed): fill, groups, reach ---------------------------------------------
     t_cal = time.time()
-    sort_scratch = torch.empty(rr.rr_sort_scratch_bytes(RR_MAX_SM_FOR_SCRATCH, 4, 1024),
-                               dtype=torch.uint8, device="cuda")   # before the region takes the rest
-    ses = Session()
+    saved_region = None
+    if args.load_calibration:
+        with open(args.load_calibration) as f:
+            saved_region = int(json.load(f).get("extra", {}).get("region_bytes", 0)) or None
+    # with a saved calibration the buffer is given the size the calibration was taken with
+    ses = Session(region_bytes=saved_region)
     N = ses.region_bytes
     fill_gbps = max(ses.fill(), ses.fill())
     loaded = None
     if args.load_calibration:
         # the layout is a property of the card: a calibration saved on this very GPU is reused
         loaded = load_calibration(args.load_calibration, ses.info["uuid"], ses.nsm, with_extra=True)
-        if loaded[3].get("region_bytes") != N:
-            raise SystemExit("bench.py: the saved calibration was taken with another buffer size")
     if loaded:
         groups, reach, grp_weights_saved, saved = loaded
         sm_reach = int(saved["sm_reach_bytes"])
@@ -326,14 +355,11 @@ def run_gpu(args):
             note="every SM's window is the whole buffer; SM cycles staggered")
         # static per-SM slices, equal work, no calibration of weights: the kernel performs each
         # warp's reads part by part of its window (same reads and checksums, another order)
-        for cached in (False, True):
-            arms["g_sorted_execution_static_per_sm_slices" + ("_cached" if cached else "")] = measure(
-                ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads,
-                           group_of_sm=owners.group_of_sm, windows=mv_windows,
-                           variant=VARIANT_SORTED, unroll=1, sort_parts=4, sort_reads=1024,
-                           sort_scratch=sort_scratch if cached else None),
-                mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
-                kernel="read_kernel<U=1, sorted>" + (", indices cached" if cached else ""))
+        arms["g_sorted_execution_static_per_sm_slices"] = measure(
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
+                       windows=mv_windows, variant=VARIANT_SORTED, unroll=1, sort_parts=4,
+                       sort_reads=1024), mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
+            kernel="read_kernel<U=1, sorted>")
     t_arms = time.time() - t_arms
     c_head = cfg4[headline]["gbps"]
     comparison = {
@@ -364,11 +390,13 @@ def run_gpu(args):
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_begin = time.time()
+        nvtx.range_push("timed")
         e0.record(stream)
         for k in range(args.steps):
             rr.rr_random_read(step_params(args.warmup + k), ses.out, ses.scratch, timed=False)
         e1.record(stream)
         torch.cuda.synchronize()
+        nvtx.range_pop()
         t_end = time.time()
         if world > 1:
             dist.barrier()
@@ -547,6 +575,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--probe-reads", type=int, default=1 << 18)
     ap.add_argument("--probe-repeats", type=int, default=3)
+    ap.add_argument("--clock-period-ms", type=int, default=50,
+                    help="period of the nvidia-smi clock sampler; 0 switches it off (do that "
+                         "under a profiler)")
     ap.add_argument("--arms", default="all", choices=["all", "headline"],
                     help="headline: only the arms value and comparison need (a, b, c at the "
                          "headline window, e)")

@@ -173,8 +173,7 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   warp's window (sort_parts equal parts): at any moment an SM then works inside 1/sort_parts of
  *   its window, which its own translation cache can hold, although the window -- the set of lines
  *   the warp may read, Section 1.3 -- is unchanged and static.  Results are those of
- *   RR_VARIANT_PACKED bit for bit; the price is sort_parts hashes per read, or, with
- *   sort_scratch, one hash and sort_parts re-reads of a cached index.
+ *   RR_VARIANT_PACKED bit for bit; the price is sort_parts hashes per read.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
@@ -214,16 +213,7 @@ typedef struct {
     uint32_t sort_parts;        /* RR_VARIANT_SORTED: parts of the window, a power of two 2..64 */
     uint32_t sort_reads;        /* RR_VARIANT_SORTED: reads per part and epoch, a multiple of  */
                                 /* 32 (1024 is a good value); both 0 for every other variant   */
-    void *sort_scratch;         /* RR_VARIANT_SORTED: DEVICE, 128-byte aligned,                */
-                                /* rr_sort_scratch_bytes() bytes, or NULL; NULL otherwise      */
 } rr_read_params_t;
-
-/* Bytes of DEVICE memory RR_VARIANT_SORTED can use to keep each warp's epoch of hashed indices
- * (nsm SMs x 32 warps x sort_parts x sort_reads x 4 bytes): with it the kernel hashes every read
- * once and re-reads the indices for each part; without it (sort_scratch = NULL) it hashes every
- * read once per part.  The contents mean nothing between calls; calls that overlap on the GPU
- * need a buffer each.                                                                          */
-size_t rr_sort_scratch_bytes(uint32_t nsm, uint32_t sort_parts, uint32_t sort_reads);
 
 typedef struct {
     double seconds_event;   /* CUDA events around the launch (0 when not timed)                */
@@ -288,8 +278,14 @@ int32_t rr_random_read_static(const rr_read_params_t *params /*HOST*/, void *out
  * random 128-byte line reads (W = 1) over the whole region with warps_per_sm warps (1..32;
  * total_reads must be a multiple of 2*warps_per_sm), warp ids and streams as in RR_MODE_PER_SM.
  * sm_a == sm_b: a solo run (total_reads/2 reads on that one SM).
- * out_dev: 2*warps_per_sm pairs {X,S}: sm_a's warps, then sm_b's (zeros for a solo run).
- * Synchronous.  res->gbps = bytes of both SMs / (latest end - earliest start, %globaltimer);
+ * The two blocks of a pair start together (the first waits at most 0.2 ms for the other), and a
+ * warp that has finished its share keeps reading its stream, 32 reads at a time, until every
+ * warp of the other SM has finished too (at most as many reads again): SMs differ in speed, and
+ * a tail in which one runs alone would dilute the contention being measured.
+ * out_dev: 2*warps_per_sm pairs {X,S} over the fixed share only: sm_a's warps, then sm_b's (zeros
+ * for a solo run).
+ * Synchronous.  res->bytes counts every line read (share and extra); res->gbps = those bytes /
+ * (latest end - earliest start, %globaltimer);
  * res->seconds_event is the event time of the launch.  RR_ERR_SM_UNCOVERED if, after three
  * launches with growing grids, one of the SMs never received a block.                        */
 int32_t rr_probe_pair(const void *buf /*DEVICE*/, uint64_t region_bytes, uint32_t sm_a,

@@ -33,7 +33,7 @@ EXPORTS = (
     "rr_gpc_map", "rr_make_weighted_windows",
     "rr_read_block_times", "rr_host_counters", "rr_probe_rate", "rr_reach_next", "rr_sm_reach",
     "rr_owner_map", "rr_phase_window", "rr_rebalance_weights", "rr_finish_spread_ppm",
-    "rr_window_cover", "rr_group_finish", "rr_probe_rows", "rr_sort_scratch_bytes",
+    "rr_window_cover", "rr_group_finish", "rr_probe_rows",
 )
 
 
@@ -65,7 +65,6 @@ class _ReadParams(ctypes.Structure):
         ("phase_reads", ctypes.c_uint32), ("mix_period", ctypes.c_uint32),
         ("phase_window_bytes", ctypes.c_uint64),
         ("sort_parts", ctypes.c_uint32), ("sort_reads", ctypes.c_uint32),
-        ("sort_scratch", ctypes.c_void_p),
     ]
 
 
@@ -143,8 +142,6 @@ def _load():
     lib.rr_probe_matrix_scratch_bytes.argtypes = [u32]
     lib.rr_probe_matrix.restype = i32
     lib.rr_probe_matrix.argtypes = [p, u64, u64, u32, u64, u32, p, u32, p, p, p, p, p]
-    lib.rr_sort_scratch_bytes.restype = ctypes.c_size_t
-    lib.rr_sort_scratch_bytes.argtypes = [u32, u32, u32]
     lib.rr_probe_rows.restype = i32
     lib.rr_probe_rows.argtypes = [p, u64, u64, u32, u64, u32, u32, u32, p, u32, p, p, p, p, p]
     lib.rr_probe_rate.restype = i32
@@ -228,10 +225,6 @@ def rr_host_counters() -> dict:
                      "device_fact_queries"), (int(x) for x in c)))
 
 
-def rr_sort_scratch_bytes(nsm: int, sort_parts: int, sort_reads: int) -> int:
-    return int(_load().rr_sort_scratch_bytes(nsm, sort_parts, sort_reads))
-
-
 def rr_scratch_bytes() -> int:
     return int(_load().rr_scratch_bytes())
 
@@ -253,7 +246,7 @@ class ReadParams:
                  group_of_sm=None, windows=None, variant: int = RR_VARIANT_LDG, unroll: int = 0,
                  warp_start=None, pool_block_reads: int = 0, phase_reads: int = 0,
                  phase_window_bytes: int = 0, mix_period: int = 0, sort_parts: int = 0,
-                 sort_reads: int = 0, sort_scratch=None):
+                 sort_reads: int = 0):
         self._groups = None
         self._windows = None
         self._warp_start = None
@@ -273,9 +266,7 @@ class ReadParams:
             self._windows.ctypes.data if self._windows is not None else None,
             n_groups, variant, unroll, pool_block_reads,
             self._warp_start.ctypes.data if self._warp_start is not None else None,
-            phase_reads, mix_period, phase_window_bytes, sort_parts, sort_reads,
-            _dev(sort_scratch) or None)
-        self._sort_scratch = sort_scratch       # keeps a tensor alive
+            phase_reads, mix_period, phase_window_bytes, sort_parts, sort_reads)
 
 
 def _result(r: _Result) -> ReadResult:

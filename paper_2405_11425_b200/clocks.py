@@ -20,6 +20,17 @@ REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_powe
 REJECTING = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
 
 
+def _die_with_parent():
+    """Runs in the child before exec: ask the kernel to end it when the parent goes away, so that
+    an aborted measurement never leaves an nvidia-smi loop behind."""
+    try:
+        import ctypes
+        import signal
+        ctypes.CDLL("libc.so.6", use_errno=True).prctl(1, signal.SIGTERM)   # PR_SET_PDEATHSIG
+    except Exception:
+        pass
+
+
 def parse_rows(rows):
     """[(unix time, sm MHz, max sm MHz, watts, {reason: bool})] from nvidia-smi CSV rows."""
     out = []
@@ -62,7 +73,7 @@ class ClockSampler:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={FIELDS}", "--format=csv,noheader,nounits",
                  "-lms", str(period_ms), "-i", str(device_index)],
-                stdout=self.file, stderr=subprocess.DEVNULL)
+                stdout=self.file, stderr=subprocess.DEVNULL, preexec_fn=_die_with_parent)
         except OSError:
             self.proc = None
 

@@ -93,12 +93,6 @@ extern "C" size_t rr_scratch_bytes(void)
     return sizeof(rr::ScratchHeader) + rr::cluster_scratch_bytes(RR_MAX_SM);
 }
 
-extern "C" size_t rr_sort_scratch_bytes(uint32_t nsm, uint32_t sort_parts, uint32_t sort_reads)
-{
-    // one epoch of 32-bit indices for each of the 32 warps a block can hold on each SM
-    return (size_t)nsm * RR_MAX_WARPS_PER_SM * sort_parts * sort_reads * sizeof(uint32_t);
-}
-
 extern "C" int32_t rr_device_info(rr_device_info_t *out, void *scratch_dev, void *stream_)
 {
     if (!out) return RR_ERR_ARG;

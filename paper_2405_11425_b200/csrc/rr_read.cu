@@ -92,7 +92,6 @@ struct ReadArgs {
     uint32_t nsm;
     uint32_t n_groups;  // 0 = ungrouped
     uint32_t pool_block;  // POOLED: smallest grab, in reads
-    uint32_t *sort_cache; // SORTED: one epoch of indices per physical warp, or null
     uint2 *out;
     ScratchHeader *scratch;
 };
@@ -102,7 +101,6 @@ constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarSorted = 3;
 // Per-warp working memory some variants need beside their registers.
 struct WarpScratch {
     uint32_t *queue;  // SORTED variant: this warp's ring of kSortQueue line indices (shared memory)
-    uint32_t *cache;  // SORTED variant: this warp's epoch of hashed indices (global), or null
 };
 constexpr uint32_t kSortQueue = 64;  // two vectors of 32 lines
 
@@ -281,30 +279,24 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
 // until 32 of them make a vector for the load loop.
 struct SortedSource {
     uint32_t *q;
-    uint32_t *cache;               // an epoch of indices, hashed once and re-read per part; or null
     uint32_t head, count;          // ring state, warp-uniform
     uint64_t epoch0, reads;        // first read of the current epoch (relative), reads of the call
     uint32_t part, batch;          // current part of the window, batch of 32 candidates inside it
     uint32_t lo, hi;               // index range of the current part
-    uint32_t ahead;                // cached mode: the index this lane looks at next (prefetched)
-    bool done, filled;
+    bool done;
     __device__ __forceinline__ void set_part(uint32_t n, uint32_t shift)
     {
         lo = (uint32_t)(((uint64_t)n * part) >> shift);
         hi = (uint32_t)(((uint64_t)n * (part + 1)) >> shift);
     }
-    __device__ __forceinline__ void init(const WarpScratch &ws, uint64_t reads_, uint32_t n,
-                                         uint32_t shift)
+    __device__ __forceinline__ void init(uint32_t *queue, uint64_t reads_, uint32_t n, uint32_t shift)
     {
-        q = ws.queue;
-        cache = ws.cache;
+        q = queue;
         head = count = 0;
         epoch0 = 0;
         reads = reads_;
         part = batch = 0;
-        ahead = 0;
         done = reads_ == 0;
-        filled = false;
         set_part(n, shift);
     }
     // Next vector of 32 lines (lane j holds the j-th); entries past the end of the call are junk.
@@ -315,43 +307,22 @@ struct SortedSource {
         const uint32_t parts = 1u << ix.sort_shift;
         const uint64_t epoch_reads = (uint64_t)ix.sort_reads << ix.sort_shift;
         while (count < 32u && !done) {
-            const uint64_t left = reads - epoch0;                       // reads from this epoch on
-            const uint64_t in_epoch = left < epoch_reads ? left : epoch_reads;
-            const uint32_t n_batches = (uint32_t)((in_epoch + 31) >> 5);
-            uint32_t idx;
-            if (cache) {
-                // Every lane writes and later re-reads its own column of the epoch only, so no
-                // ordering between lanes is needed; .cg keeps the column out of L1.
-                if (!filled) {
-                    for (uint32_t b = 0; b < n_batches; ++b) {
-                        const uint64_t t = epoch0 + ((uint64_t)b << 5) + lane;
-                        const uint32_t v = t < reads
-                                               ? mod_exact(sm64(key + (first + t) * kGamma), div)
-                                               : 0xFFFFFFFFu;  // beyond the call: in no part
-                        __stcg(cache + (b << 5) + lane, v);
-                    }
-                    filled = true;
-                    ahead = __ldcg(cache + lane);
-                }
-                idx = ahead;
-                const uint32_t nb = batch + 1 < n_batches ? batch + 1 : 0;
-                ahead = __ldcg(cache + (nb << 5) + lane);
-            } else {
-                const uint64_t t = epoch0 + ((uint64_t)batch << 5) + lane;   // relative read index
-                idx = t < reads ? mod_exact(sm64(key + (first + t) * kGamma), div) : 0xFFFFFFFFu;
-            }
-            const bool keep = idx >= lo && idx < hi;
+            const uint64_t t = epoch0 + ((uint64_t)batch << 5) + lane;   // relative read index
+            const uint32_t idx = mod_exact(sm64(key + (first + t) * kGamma), div);
+            const bool keep = t < reads && idx >= lo && idx < hi;
             const uint32_t m = __ballot_sync(0xFFFFFFFFu, keep);
             if (keep) q[(head + count + __popc(m & ((1u << lane) - 1u))) & (kSortQueue - 1)] = base + idx;
             count += __popc(m);
             // advance: next batch of this part, else next part, else next epoch
-            if (++batch >= n_batches) {
+            ++batch;
+            const uint64_t left = reads - epoch0;                       // reads from this epoch on
+            const uint64_t in_epoch = left < epoch_reads ? left : epoch_reads;
+            if (((uint64_t)batch << 5) >= in_epoch) {
                 batch = 0;
                 if (++part == parts) {
                     part = 0;
                     epoch0 += in_epoch;
                     done = epoch0 >= reads;
-                    filled = false;
                 }
                 set_part(n, ix.sort_shift);
             }
@@ -378,7 +349,7 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
     static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a vector");
     const Divisor div = make_divisor(n);
     SortedSource src;
-    src.init(br, reads, n, ix.sort_shift);
+    src.init(br.queue, reads, n, ix.sort_shift);
     const uint32_t sub = lane / NL;
     const char *lane_ptr = buf + (lane % NL) * 16u;
     uint32_t d[U][4];
@@ -450,17 +421,10 @@ __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_
                                                    base, n, lane, X, S, violations);
 }
 
-// Where physical warp number `slot` of the grid keeps its epoch of indices.
-__device__ __forceinline__ uint32_t *sort_cache_of(const ReadArgs &a, uint32_t slot)
-{
-    return a.sort_cache ? a.sort_cache + (size_t)slot * ((size_t)a.ix.sort_reads << a.ix.sort_shift)
-                        : nullptr;
-}
-
 template <int VAR>
 __device__ __forceinline__ WarpScratch make_warp_scratch(uint32_t warp)
 {
-    WarpScratch ws{nullptr, nullptr};
+    WarpScratch ws{nullptr};
     if constexpr (VAR == kVarSorted) {
         __shared__ uint32_t sh_sort_queue[32 * kSortQueue];
         ws.queue = sh_sort_queue + warp * kSortQueue;
@@ -495,7 +459,6 @@ __global__ void __launch_bounds__(1024, 1)
         if (slot >= a.cps) return;
         const uint32_t g = sh_group[sm];
         if (g == RR_SM_INACTIVE) return;
-        br.cache = sort_cache_of(a, (sm * a.cps + slot) * a.wpc + warp);
         const uint32_t base = sh_win[g].base_line, n = sh_win[g].n_lines;
         const uint32_t v0 = tab.warp_start[g], cnt = tab.warp_start[g + 1] - v0;
         // physical warps working for this group: its SMs times the warps of one block
@@ -567,7 +530,6 @@ __global__ void __launch_bounds__(1024, 1)
         __syncthreads();
         const uint32_t sm = sh_sm, slot = sh_slot;
         if (slot >= a.cps) return;  // not among the first blocks on this SM
-        br.cache = sort_cache_of(a, (sm * a.cps + slot) * a.wpc + warp);
         uint32_t base = 0, n = a.n_lines;
         if (a.n_groups) {
             const uint32_t g = sh_group[sm];
@@ -600,7 +562,6 @@ __global__ void __launch_bounds__(1024, 1)
         uint64_t t_start = 0;
         if (threadIdx.x == 0) t_start = globaltimer();
         const uint64_t stride = (uint64_t)gridDim.x * a.wpc;
-        br.cache = sort_cache_of(a, blockIdx.x * a.wpc + warp);
         for (uint64_t v = (uint64_t)blockIdx.x * a.wpc + warp; v < a.n_warps; v += stride) {
             uint32_t X, S;
             warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
@@ -637,7 +598,7 @@ struct ProbeArgs {
 constexpr int kProbeUnroll = 8;
 constexpr uint32_t kProbeRendezvousPolls = 1u << 16;  // both limits bound the wait at the start
 constexpr uint64_t kProbeRendezvousNs = 200000;       // 0.2 ms
-constexpr uint32_t kProbeExtraChunk = 64;             // reads between two looks at the other SM
+constexpr uint32_t kProbeExtraChunk = 32;             // reads between two looks at the other SM
 
 __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ ProbeArgs a)
 {
@@ -673,7 +634,7 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
     const uint64_t key = sm64(a.key_seed ^ v), V = (uint64_t)a.nsm * a.wps;
     const IndexSpec ix{RR_INDEX_RANDOM, 0u, 0u, 0u, 0u, 0u, 0u};
     uint32_t X, S;
-    WarpScratch no_ring{nullptr, nullptr};
+    WarpScratch no_ring{nullptr};
     warp_reads<1, kProbeUnroll, kVarLdg>(a.buf, a.region_bytes, key, ix, v, V, 0, a.reads, 0u,
                                          a.n_lines, lane, X, S, nullptr, no_ring);
     if (lane == 0) {
@@ -778,8 +739,7 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
         const uint32_t P = p->sort_parts, R = p->sort_reads;
         if (p->words_per_lane == 4 || p->index_mode != RR_INDEX_RANDOM) return RR_ERR_ARG;
         if (P < 2 || P > 64 || (P & (P - 1)) || R < 32 || R % 32u || R > (1u << 20)) return RR_ERR_ARG;
-        if ((uintptr_t)p->sort_scratch % 128u) return RR_ERR_ALIGN;
-    } else if (p->sort_parts || p->sort_reads || p->sort_scratch) {
+    } else if (p->sort_parts || p->sort_reads) {
         return RR_ERR_ARG;
     }
     if (p->index_mode == RR_INDEX_MIXED) {
@@ -1017,7 +977,6 @@ static void make_launch_args(const rr_read_params_t *p, const Geometry &g, const
     a->nsm = (uint32_t)f.nsm;
     a->n_groups = p->group_of_sm ? p->n_groups : 0;
     a->pool_block = p->pool_block_reads ? p->pool_block_reads : 64u;
-    a->sort_cache = p->variant == RR_VARIANT_SORTED ? (uint32_t *)p->sort_scratch : nullptr;
     a->out = (uint2 *)out_dev;
     a->scratch = (ScratchHeader *)scratch_dev;
     std::memset(tab, 0, sizeof(*tab));

@@ -224,17 +224,14 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     R["moving_windows_no_partition"] = moving_all
 
     # sorted execution: the same static per-SM slices, equal work, each warp's reads taken part by
-    # part of its window -- hashing once per part, or once with the indices kept in a scratch
+    # part of its window (the indices are hashed once per part)
     sorted_rows = []
     for parts in (2, 4, 8):
-        cache = torch.empty(rr.rr_sort_scratch_bytes(ses.nsm, parts, 1024), dtype=torch.uint8,
-                            device="cuda")
-        for cached in (False, True):
+        for U in (1, 2):
             d = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=owners_eq.group_of_sm,
-                       windows=eq_win, variant=rr.RR_VARIANT_SORTED, unroll=1, sort_parts=parts,
-                       sort_reads=1024, sort_scratch=cache if cached else None)
-            sorted_rows.append({"parts": parts, "cached": cached, **d})
-        del cache
+                       windows=eq_win, variant=rr.RR_VARIANT_SORTED, unroll=U, sort_parts=parts,
+                       sort_reads=1024)
+            sorted_rows.append({"parts": parts, "unroll": U, **d})
     R["sorted_execution"] = sorted_rows
 
     # work in proportion to group capacity (pooled mode), balanced under sustained load
@@ -363,10 +360,9 @@ def markdown(R: dict) -> str:
     L.append("")
     if "sorted_execution" in R:
         L += ["## Sorted execution: static per-SM slices, equal work, reads taken part by part", "",
-              "| parts | indices | GB/s |", "|---|---|---|"]
+              "| parts | warp loads in flight | GB/s |", "|---|---|---|"]
         for r in R["sorted_execution"]:
-            L.append(f"| {r['parts']} | {'hashed once, cached' if r['cached'] else 'hashed per part'} "
-                     f"| {f(r)} |")
+            L.append(f"| {r['parts']} | {r['unroll']} | {f(r)} |")
         L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]

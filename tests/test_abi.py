@@ -69,9 +69,6 @@ def test_read_argument_errors_come_before_any_cuda_call():
     assert _call(**{**srt, "index_mode": rr.RR_INDEX_STRIDE}) == rr.RR_ERR_ARG
     assert _call(**{**srt, "unroll": 8}) == rr.RR_ERR_ARG
     assert _call(sort_parts=4) == rr.RR_ERR_ARG                              # only with SORTED
-    assert _call(sort_scratch=FAKE) == rr.RR_ERR_ARG
-    assert _call(**{**srt, "sort_scratch": FAKE + 64}) == rr.RR_ERR_ALIGN
-    assert rr.rr_sort_scratch_bytes(148, 4, 1024) == 148 * 32 * 4096 * 4
     assert _call(variant=9) == rr.RR_ERR_ARG
     assert _call(unroll=3) == rr.RR_ERR_ARG
     assert _call(n_warps=0) == rr.RR_ERR_ARG

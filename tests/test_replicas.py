@@ -74,10 +74,16 @@ def test_calibration_round_trip_is_bound_to_the_card(tmp_path):
     g = Groups(np.array([0, 0, 1, 1, 2, 2], np.uint16), 3, 47.0)
     r = Reach(True, 4600.0, 70 << 30, [(1 << 30, 5400.0)])
     path = tmp_path / "card.json"
-    save_calibration(path, "abc123", g, r, weights=[5, 6, 7])
+    g.probe_stats = {"overlap_min": 0.985, "pairs_below_goal": 0, "reruns": 0, "relaunched": 0}
+    save_calibration(path, "abc123", g, r, weights=[5, 6, 7],
+                     extra={"region_bytes": 123 << 20, "weights_per_window": [1, 2, 3, 4, 5, 6]})
     g2, r2, w2 = load_calibration(path, "abc123", 6)
     assert np.array_equal(g2.group_of_sm, g.group_of_sm) and g2.n_groups == 3 and g2.sizes == [2, 2, 2]
     assert r2.cliff and r2.reach_bytes == 70 << 30 and list(w2) == [5, 6, 7]
+    assert r2.sweep == [(1 << 30, 5400.0)] and g2.overlap_min == 0.985
+    g3, r3, w3, extra = load_calibration(path, "abc123", 6, with_extra=True)
+    assert extra["region_bytes"] == 123 << 20 and extra["weights_per_window"] == [1, 2, 3, 4, 5, 6]
+    assert g3.probe_stats["pairs_below_goal"] == 0
     with pytest.raises(ValueError):
         load_calibration(path, "another-card", 6)
     with pytest.raises(ValueError):
