@@ -59,9 +59,11 @@ SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
 NSM_NOMINAL = 148
-# DRAM bytes moved per algorithmic byte by the read kernel, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over lines x 128 B, 4 GiB case).
-TRAFFIC_PER_ALGORITHMIC_BYTE = 0.975
+# DRAM bytes moved per algorithmic byte by the read kernel: dram__bytes_read.sum +
+# dram__bytes_write.sum over lines x 128 B, from the one-pass ncu capture of the same kernel and
+# plan shape on a 160 GiB region that is summarised in profiles/ (9.93 GB read + 0.004 GB written
+# per 9.932 GB launch; on a 4 GiB region L2 hits bring it down to 0.976).
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0
 
 
 def _peaks():
@@ -523,7 +525,8 @@ def _run_gpu(args, holder):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind} (copy, read+write)",
                          "traffic": TRAFFIC_PER_ALGORITHMIC_BYTE * step_bytes,
-                         "traffic_kind": "scaled from the 4 GiB ncu capture by lines read",
+                         "traffic_kind": "scaled by lines read from the one-pass ncu capture of the "
+                                         "same kernel on a 160 GiB region (16384 reads per warp)",
                          "theoretical_gbps": ses.info["theoretical_gbps"],
                          "frac_of_theoretical": achieved / ses.info["theoretical_gbps"]},
             "cpu_baseline": cpu,

@@ -341,7 +341,7 @@ template <int W, int U>
 __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, uint64_t key,
                                                   IndexSpec ix, uint64_t first, uint64_t reads,
                                                   uint32_t base, uint32_t n, uint32_t lane,
-                                                  uint32_t &X, uint32_t &S, WarpScratch &br)
+                                                  uint32_t &X, uint32_t &S, WarpScratch &ws)
 {
     constexpr int P = 4 / W;     // lines per warp load
     constexpr int NL = 32 / P;   // warp loads per vector of 32 lines = lanes per line
@@ -349,7 +349,7 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
     static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a vector");
     const Divisor div = make_divisor(n);
     SortedSource src;
-    src.init(br.queue, reads, n, ix.sort_shift);
+    src.init(ws.queue, reads, n, ix.sort_shift);
     const uint32_t sub = lane / NL;
     const char *lane_ptr = buf + (lane % NL) * 16u;
     uint32_t d[U][4];
@@ -410,12 +410,12 @@ __device__ __forceinline__ void warp_reads(const char *__restrict__ buf, uint64_
                                            uint64_t key, IndexSpec ix, uint64_t v,
                                            uint64_t V, uint64_t first, uint64_t reads,
                                            uint32_t base, uint32_t n, uint32_t lane, uint32_t &X,
-                                           uint32_t &S, uint32_t *violations, WarpScratch &br)
+                                           uint32_t &S, uint32_t *violations, WarpScratch &ws)
 {
     if constexpr (VAR == kVarPacked && W < 4)
         warp_reads_packed<W, U>(buf, key, ix, v, V, first, reads, base, n, lane, X, S);
     else if constexpr (VAR == kVarSorted && W < 4)
-        warp_reads_sorted<W, U>(buf, key, ix, first, reads, base, n, lane, X, S, br);
+        warp_reads_sorted<W, U>(buf, key, ix, first, reads, base, n, lane, X, S, ws);
     else
         warp_reads_lines<W, U, VAR == kVarChecked>(buf, region_bytes, key, ix, v, V, first, reads,
                                                    base, n, lane, X, S, violations);
@@ -441,7 +441,7 @@ __global__ void __launch_bounds__(1024, 1)
     __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     ScratchHeader *sc = a.scratch;
-    WarpScratch br = make_warp_scratch<VAR>(warp);
+    WarpScratch ws = make_warp_scratch<VAR>(warp);
 
     if (a.mode == RR_MODE_POOLED) {
         // Work sharing inside an SM group: items (logical warp, block of reads) come from the
@@ -500,7 +500,7 @@ __global__ void __launch_bounds__(1024, 1)
                 uint32_t X, S;
                 warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix,
                                           v, a.n_warps, a.first_read + i0, n_seg, base, n, lane, X,
-                                          S, &sc->violations, br);
+                                          S, &sc->violations, ws);
                 if (lane == 0) {
                     atomicXor(&out_words[2 * v], X);
                     atomicAdd(&out_words[2 * v + 1], S);
@@ -546,7 +546,7 @@ __global__ void __launch_bounds__(1024, 1)
         ix.sm = sm;
         ix.nsm = a.nsm;
         warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), ix, v, V, a.first_read,
-                              a.reads, base, n, lane, X, S, &sc->violations, br);
+                              a.reads, base, n, lane, X, S, &sc->violations, ws);
         if (lane == 0) a.out[v] = make_uint2(X, S);
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -566,7 +566,7 @@ __global__ void __launch_bounds__(1024, 1)
             uint32_t X, S;
             warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
                                       a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
-                                      &sc->violations, br);
+                                      &sc->violations, ws);
             if (lane == 0) a.out[v] = make_uint2(X, S);
         }
         __syncthreads();

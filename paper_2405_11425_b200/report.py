@@ -30,6 +30,10 @@ from .pipeline import GiB, Session
 def _stats(ses, region, reps=5, *, settle=30, min_ms=50.0, **kw):
     """One figure of the report: Session.sustained (settling launches, then `reps` regions of at
     least `min_ms` of back-to-back launches), median / min / max GB/s."""
+    if "variant" not in kw:          # the packed shape wherever it exists (W = 1, 2), as bench.py
+        packed = kw.get("W", 1) < 4
+        kw["variant"] = rr.RR_VARIANT_PACKED if packed else rr.RR_VARIANT_LDG
+        kw.setdefault("unroll", 2 if packed else 8)
     d = ses.sustained(ses.params(region, **kw), settle=settle, min_ms=min_ms, reps=reps)
     return {"median": d["gbps"], "min": d["gbps_min"], "max": d["gbps_max"]}
 
