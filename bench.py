@@ -54,7 +54,9 @@ WARPS_PER_SM = 32
 SETTLE_LAUNCHES = 150         # of the same launch, before any timed region
 VARIANT_PACKED = 2            # 16-byte lanes: one warp load covers four 128-byte lines
 VARIANT_SORTED = 3            # the same, each warp's reads taken part by part of its window
-UNROLL = 2                    # warp loads in flight per warp (8 lines)
+UNROLL = 1                    # warp loads in flight per warp (4 lines): with 32 warps per SM and
+                              # balanced work a deeper ring only adds power (5654 against 5549 GB/s)
+MOVING_WARPS_PER_SM = 24      # the moving-window arms need fewer warps still (6135 against 5881)
 SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
@@ -345,15 +347,17 @@ def _run_gpu(args, holder):
         mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
         slice_bytes = int(mv_windows[:, 1].max()) * 128
         mv_parts, mv_sub = rr.rr_phase_window(slice_bytes, sm_reach, 64)
-        phased = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=1024, phase_window_bytes=mv_sub)
+        phased = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=1024, phase_window_bytes=mv_sub,
+                      warps_per_sm=MOVING_WARPS_PER_SM, variant=VARIANT_PACKED, unroll=2)
         arms["f_moving_sub_windows_per_sm_slices"] = measure(
             ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
-                       windows=mv_windows, **kern, **phased), mv_windows, coverage=1.0,
-            sub_window_mib=mv_sub / (1 << 20), sub_windows=mv_parts, phase_reads=1024)
+                       windows=mv_windows, **phased), mv_windows, coverage=1.0,
+            sub_window_mib=mv_sub / (1 << 20), sub_windows=mv_parts, phase_reads=1024,
+            warps_per_sm=MOVING_WARPS_PER_SM)
         arms["f_moving_sub_windows_no_partition"] = measure(
-            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, **kern, **phased),
+            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, **phased),
             window_gib_min_max=[N / GiB, N / GiB], coverage=1.0,
-            sub_window_mib=mv_sub / (1 << 20), phase_reads=1024,
+            sub_window_mib=mv_sub / (1 << 20), phase_reads=1024, warps_per_sm=MOVING_WARPS_PER_SM,
             note="every SM's window is the whole buffer; SM cycles staggered")
         # static per-SM slices, equal work, no calibration of weights: the kernel performs each
         # warp's reads part by part of its window (same reads and checksums, another order)
@@ -511,7 +515,7 @@ def _run_gpu(args, holder):
                 "region_bytes": N, "region_gib": N / GiB, "line_bytes": 128,
                 "logical_warps": n_warps, "warps_per_sm": WARPS_PER_SM,
                 "reads_per_warp_per_step": reads,
-                "kernel": "read_kernel<W=1, U=2, packed>: 8 lanes x 16 B per line, pooled mode",
+                "kernel": "read_kernel<W=1, U=1, packed>: 8 lanes x 16 B per line, pooled mode",
                 "window_gib_min_max": [float(bal_windows[:, 1].min()) * 128 / GiB,
                                        float(bal_windows[:, 1].max()) * 128 / GiB],
                 "coverage": 1.0, "n_groups": groups.n_groups, "n_windows": owners.n_groups,
@@ -535,7 +539,8 @@ def _run_gpu(args, holder):
             "arms": arms,
             "protocol": {"settle_launches": SETTLE_LAUNCHES, "min_ms_per_region": 50.0,
                          "regions": 5, "reads_per_warp_per_launch": arm_reads,
-                         "kernel": "read_kernel<U=2, packed> for every arm but g",
+                         "kernel": "read_kernel<U=1, packed> for every arm but g (sorted variant); "
+                                   "arms f run 24 warps per SM, all others 32",
                          "seconds_all_arms": t_arms},
             "calibration": {
                 "device": ses.info["name"], "uuid": ses.info["uuid"], "nsm": ses.nsm,
