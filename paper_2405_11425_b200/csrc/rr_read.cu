@@ -47,6 +47,23 @@ __device__ __forceinline__ uint64_t draw_index(const IndexSpec &ix, uint64_t key
     return sm64(key + i * kGamma);
 }
 
+// The same for a lane that walks its warp's stream 32 reads at a time (read i, then i + 32, ...):
+// the generator state key + i * gamma is carried along and advanced by one addition, and the
+// purely random modes never look at the sequential rules.
+struct LaneStream {
+    uint64_t state;  // key + i * gamma for the lane's next read
+    __device__ __forceinline__ void init(uint64_t key, uint64_t i) { state = key + i * kGamma; }
+    __device__ __forceinline__ uint64_t next(const IndexSpec &ix, uint64_t key, uint64_t i,
+                                             uint64_t v, uint64_t V)
+    {
+        // RANDOM and PHASED: every read is a hash of the state
+        const bool random = ix.mode == RR_INDEX_RANDOM || ix.mode == RR_INDEX_PHASED;
+        const uint64_t r = random ? sm64(state) : draw_index(ix, key, i, v, V);
+        state += 32u * kGamma;
+        return r;
+    }
+};
+
 // The window a batch of 32 reads draws from: the warp's whole window, or (PHASED) the
 // sub-window of the batch's phase.  Recomputed only when the phase changes.
 struct LineSource {
@@ -118,8 +135,10 @@ __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, u
     uint32_t d[U][W];
     uint32_t x = 0, s = 0;
 
-    auto gen = [&](uint64_t i) -> uint32_t {
-        const uint64_t r = draw_index(ix, key, i, v, V);
+    LaneStream stream;
+    stream.init(key, first + lane);
+    auto gen = [&](uint64_t i) -> uint32_t {  // called for i = first + lane, then + 32 each time
+        const uint64_t r = stream.next(ix, key, i, v, V);
         return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[W]) {
@@ -211,8 +230,10 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
     uint32_t d[U][4];
     uint32_t x = 0, s = 0;
 
-    auto gen = [&](uint64_t i) -> uint32_t {
-        const uint64_t r = draw_index(ix, key, i, v, V);
+    LaneStream stream;
+    stream.init(key, first + lane);
+    auto gen = [&](uint64_t i) -> uint32_t {  // called for i = first + lane, then + 32 each time
+        const uint64_t r = stream.next(ix, key, i, v, V);
         return src.base + mod_exact(r, src.div);
     };
     auto issue = [&](uint32_t line, uint32_t(&dst)[4]) {
