@@ -192,24 +192,44 @@ def test_pooled_bench_launch_configuration_sampled(ses):
 
 
 def test_pooled_one_window_per_sm_sampled(ses):
-    # bench.py's owner map: one window per SM (148 "groups"), weights differing per SM
+    # bench.py's timed step: one window per SM (148 "groups"), weights differing per SM, 2^19
+    # reads per warp continuing the stream at a late first_read, one warp load in flight per warp
     region = ses.region_bytes
     rng = np.random.default_rng(3)
     owners = rng.permutation(ses.nsm).astype(np.uint16)
     weights = rng.integers(5000, 8000, ses.nsm)
     n_warps = ses.nsm * WPS
     win, ws = rr.rr_make_weighted_windows(region, 1, weights, n_warps, max_window_bytes=64 * GiB)
-    reads = 256 * 64
+    reads, first = 1 << 19, 24 << 19
     p = ses.params(region, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps, warps_per_sm=WPS,
-                   reads_per_warp=reads, seed=rr_inputs.CFG4_SEED, group_of_sm=owners, windows=win,
-                   warp_start=ws, variant=rr.RR_VARIANT_PACKED, unroll=2)
-    res = rr.rr_random_read(p, ses.out, ses.scratch)
-    assert res.sms_covered == ses.nsm
+                   reads_per_warp=reads, first_read=first, seed=rr_inputs.CFG4_SEED,
+                   group_of_sm=owners, windows=win, warp_start=ws, variant=rr.RR_VARIANT_PACKED,
+                   unroll=1)
+    assert rr.rr_random_read(p, ses.out, ses.scratch, timed=False) is None   # as bench launches it
+    res = rr.rr_read_report(p, ses.scratch)
+    assert res.sms_covered == ses.nsm and res.bytes == n_warps * reads * 128
     got = ses.checksums(n_warps)
-    for v in _sample(n_warps):
+    for v in _sample(n_warps)[::3]:
         g = int(np.searchsorted(ws, v, side="right") - 1)
         base, n = map(int, win[g])
-        assert tuple(got[v]) == oracle.warp_checksum(rr_inputs.CFG4_SEED, v, 0, reads, 1, base, n), v
+        assert tuple(got[v]) == oracle.warp_checksum(rr_inputs.CFG4_SEED, v, first, reads, 1, base,
+                                                     n), v
+
+
+def test_sorted_execution_over_the_whole_buffer_sampled(ses):
+    # bench.py's arm g: one static slice per SM, equal work, each warp's reads taken in epochs of
+    # 4 x 1024, part by part of its 1.1 GiB window
+    region = ses.region_bytes
+    owners = np.arange(ses.nsm, dtype=np.uint16)[::-1].copy()
+    win, _ = rr.rr_make_weighted_windows(region, 1, [1] * ses.nsm, ses.nsm * WPS)
+    reads, first = 256 * 64 + 77, 4096 * 3           # a ragged last epoch
+    p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=reads, first_read=first,
+                   seed=rr_inputs.CFG4_SEED, group_of_sm=owners, windows=win,
+                   variant=rr.RR_VARIANT_SORTED, unroll=1, sort_parts=4, sort_reads=1024)
+    res = rr.rr_random_read(p, ses.out, ses.scratch)
+    assert res.sms_covered == ses.nsm and res.bytes == ses.nsm * WPS * reads * 128
+    _check_sampled(ses, ses.checksums(ses.nsm * WPS), region, 1, reads, rr_inputs.CFG4_SEED,
+                   owners, win, first)
 
 
 def test_balancing_loop_yields_a_valid_plan_and_exact_checksums(ses):
