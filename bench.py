@@ -297,6 +297,11 @@ def _run_gpu(args, holder):
         arms["c3_naive_per_sm_control"] = measure(
             ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=ctrl_groups,
                        windows=ctrl_win, **kern), ctrl_win, coverage=ctrl_cov)
+        pw_win, pw_cov = rr.rr_make_windows(N, 1, S, 256, policy=1, seed=SEED)
+        arms["c4_naive_per_warp_control"] = measure(
+            ses.params(N, W=1, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps, seed=SEED,
+                       reads_per_warp=arm_reads, windows=pw_win, **kern), pw_win, coverage=pw_cov,
+            note="warp v reads inside hashed chunk v mod 256, whatever SM runs it")
         ov_win, ov_cov = rr.rr_make_windows(N, 1, S, groups.n_groups, policy=2)
         covered, dmin, dmax = rr.rr_window_cover(ov_win, N // 128)
         arms["c_overlapping_windows_per_group"] = measure(

@@ -140,7 +140,10 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *
  * The region is the prefix [0, region_bytes) of buf; L = floor(region_bytes / (128*W)) lines.
  * RR_MODE_LOGICAL: n_warps logical warps, each reading the whole region; any block may run
- *   any warp; out has n_warps entries.
+ *   any warp; out has n_warps entries.  With windows[n_groups] (HOST) and no group_of_sm, warp v
+ *   reads inside windows[v mod n_groups] instead: a window chosen per warp with no regard for SMs
+ *   -- the naive control of Section 2.1 one level finer than per SM (use rr_make_windows
+ *   policy 1 for the windows).
  * RR_MODE_PER_SM: a persistent grid, warps_per_sm warps on every SM; a block reads %smid,
  *   claims the SM, looks its group and window up in a table in shared memory; warp
  *   v = smid*warps_per_sm + w.  group_of_sm == NULL: every SM active, window = whole region.

@@ -74,6 +74,8 @@ def _load():
         lib.orc_warp_checksum_mixed.argtypes = [u64, u64, u64, u64, u64, u32, u64, u64, u64, p, p]
         lib.orc_read_per_sm_mixed.restype = i32
         lib.orc_read_per_sm_mixed.argtypes = [u64, u32, u32, u32, u64, u64, u64, p, p, p, u32, u64, p]
+        lib.orc_read_logical_windows.restype = i32
+        lib.orc_read_logical_windows.argtypes = [u64, u32, u64, u64, u64, u64, p, p, u32, p]
         lib.orc_read_logical.restype = i32
         lib.orc_read_logical.argtypes = [u64, u32, u32, u64, u64, u64, u64, p]
         lib.orc_read_logical_materialised.restype = i32
@@ -164,6 +166,20 @@ def read_logical(region_bytes: int, W: int, n_warps: int, reads: int, seed: int,
     out = np.zeros((n_warps, 2), dtype=np.uint32)
     rc = _load().orc_read_logical(region_bytes, W, index_mode, n_warps, first_read, reads, seed,
                                   _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
+
+
+def read_logical_windows(region_bytes: int, W: int, n_warps: int, reads: int, seed: int, windows,
+                         first_read: int = 0) -> np.ndarray:
+    """Logical warps 0..n_warps-1, warp v inside window v mod len(windows)."""
+    w = np.ascontiguousarray(windows, dtype=np.uint32).reshape(-1, 2)
+    wb = np.ascontiguousarray(w[:, 0])
+    wn = np.ascontiguousarray(w[:, 1])
+    out = np.zeros((n_warps, 2), dtype=np.uint32)
+    rc = _load().orc_read_logical_windows(region_bytes, W, n_warps, first_read, reads, seed,
+                                          _ptr(wb), _ptr(wn), w.shape[0], _ptr(out))
     if rc != 0:
         raise OracleError(rc)
     return out

@@ -324,6 +324,30 @@ int32_t orc_read_logical(uint64_t region_bytes, uint32_t W, uint32_t index_mode,
     return ORC_OK;
 }
 
+/* Logical-warp mode with a window per warp: warp v reads inside window v mod n_windows.
+ * Section 2.1 tries the simplest restriction first -- every SM on its own random half --
+ * and finds no benefit; this is the same control one level finer, a window chosen per
+ * warp with no regard for SMs or groups (windows from orc_make_windows policy 1).       */
+int32_t orc_read_logical_windows(uint64_t region_bytes, uint32_t W, uint64_t n_warps,
+                                 uint64_t first_read, uint64_t reads, uint64_t seed,
+                                 const uint32_t *win_base, const uint32_t *win_n,
+                                 uint32_t n_windows, uint32_t *out)
+{
+    if (!orc_width_ok(W) || !out || !win_base || !win_n || n_windows == 0) return ORC_ERR_ARG;
+    uint64_t L = region_bytes / (128ull * W);
+    if (L == 0 || L > 0xFFFFFFFFull) return ORC_ERR_RANGE;
+    for (uint32_t g = 0; g < n_windows; ++g)
+        if (win_n[g] == 0 || (uint64_t)win_base[g] + win_n[g] > L) return ORC_ERR_RANGE;
+    int64_t nw = (int64_t)n_warps;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t v = 0; v < nw; ++v) {
+        uint32_t g = (uint32_t)((uint64_t)v % n_windows);
+        orc_warp_checksum(ORC_INDEX_RANDOM, seed, (uint64_t)v, n_warps, first_read, reads, W,
+                          win_base[g], win_n[g], &out[2 * v], &out[2 * v + 1]);
+    }
+    return ORC_OK;
+}
+
 /* Per-SM mode: v = smid*wps + warp; window = windows[group_of_sm[smid]] (whole
  * region when group_of_sm is NULL); inactive SMs (0xFFFF) give {0,0}.
  * out holds nsm*wps pairs.                                                      */

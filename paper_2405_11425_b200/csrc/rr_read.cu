@@ -580,13 +580,23 @@ __global__ void __launch_bounds__(1024, 1)
             atomicAdd(&sc->blocks_run, 1u);
         }
     } else {
+        if (a.n_groups) {  // a window per warp: warp v reads inside windows[v mod n_groups]
+            for (uint32_t k = threadIdx.x; k < a.n_groups; k += blockDim.x) sh_win[k] = tab.windows[k];
+            __syncthreads();
+        }
         uint64_t t_start = 0;
         if (threadIdx.x == 0) t_start = globaltimer();
         const uint64_t stride = (uint64_t)gridDim.x * a.wpc;
         for (uint64_t v = (uint64_t)blockIdx.x * a.wpc + warp; v < a.n_warps; v += stride) {
+            uint32_t base = 0, n = a.n_lines;
+            if (a.n_groups) {
+                const rr_window_t w = sh_win[v % a.n_groups];
+                base = w.base_line;
+                n = w.n_lines;
+            }
             uint32_t X, S;
             warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
-                                      a.n_warps, a.first_read, a.reads, 0u, a.n_lines, lane, X, S,
+                                      a.n_warps, a.first_read, a.reads, base, n, lane, X, S,
                                       &sc->violations, ws);
             if (lane == 0) a.out[v] = make_uint2(X, S);
         }
@@ -789,7 +799,16 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     if (L == 0 || L > 0xFFFFFFFFull) return RR_ERR_RANGE;
     if (p->reads_per_warp > (1ull << 62) || p->first_read > (1ull << 62)) return RR_ERR_RANGE;
     if (p->mode == RR_MODE_LOGICAL) {
-        if (p->n_warps == 0 || p->group_of_sm || p->windows || p->n_groups) return RR_ERR_ARG;
+        if (p->n_warps == 0 || p->group_of_sm) return RR_ERR_ARG;
+        if (p->windows) {  // a window per warp
+            if (p->n_groups == 0 || p->n_groups > RR_MAX_GROUPS) return RR_ERR_ARG;
+            for (uint32_t g = 0; g < p->n_groups; ++g)
+                if (p->windows[g].n_lines == 0 ||
+                    (uint64_t)p->windows[g].base_line + p->windows[g].n_lines > L)
+                    return RR_ERR_RANGE;
+        } else if (p->n_groups) {
+            return RR_ERR_ARG;
+        }
     } else if (p->mode == RR_MODE_POOLED) {
         const uint32_t w = p->warps_per_sm;
         if (w == 0 || w > RR_MAX_WARPS_PER_SM || p->nsm == 0 || p->nsm > RR_MAX_SM) return RR_ERR_ARG;
@@ -996,15 +1015,13 @@ static void make_launch_args(const rr_read_params_t *p, const Geometry &g, const
     a->wpc = g.wpc;
     a->cps = g.cps;
     a->nsm = (uint32_t)f.nsm;
-    a->n_groups = p->group_of_sm ? p->n_groups : 0;
+    a->n_groups = p->windows ? p->n_groups : 0;
     a->pool_block = p->pool_block_reads ? p->pool_block_reads : 64u;
     a->out = (uint2 *)out_dev;
     a->scratch = (ScratchHeader *)scratch_dev;
     std::memset(tab, 0, sizeof(*tab));
-    if (p->group_of_sm) {
-        std::memcpy(tab->group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
-        std::memcpy(tab->windows, p->windows, sizeof(rr_window_t) * p->n_groups);
-    }
+    if (p->group_of_sm) std::memcpy(tab->group_of_sm, p->group_of_sm, sizeof(uint16_t) * f.nsm);
+    if (p->windows) std::memcpy(tab->windows, p->windows, sizeof(rr_window_t) * p->n_groups);
     if (p->mode == RR_MODE_POOLED)
         std::memcpy(tab->warp_start, p->warp_start, sizeof(uint32_t) * (p->n_groups + 1));
 }

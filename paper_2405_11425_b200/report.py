@@ -156,6 +156,11 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
             rows[name]["naive_per_sm_control"] = _stats(ses, N, reps, W=W, seed=23,
                                                         reads_per_warp=reads, group_of_sm=cg,
                                                         windows=cw)
+            # the same control one level finer: a hashed chunk per warp, whatever SM runs it
+            pw, _ = rr.rr_make_windows(N, W, S_w, 256, policy=1, seed=23)
+            rows[name]["naive_per_warp_control"] = _stats(
+                ses, N, reps, W=W, seed=23, reads_per_warp=reads, mode=rr.RR_MODE_LOGICAL,
+                n_warps=ses.nsm * 32, windows=pw)
             # windows of the same size, evenly spaced and overlapping (policy 2)
             ow, ocov = rr.rr_make_windows(N, W, S_w, groups.n_groups, policy=2)
             covered, dmin, dmax = rr.rr_window_cover(ow, N // (128 * W))
@@ -337,13 +342,14 @@ def markdown(R: dict) -> str:
     for width, d in R["cfg4_grouped"].items():
         L += [f"### {width} lines: unrestricted over everything {f(d['unrestricted_full'])}", "",
               "| window | GiB | coverage | grouped | unrestricted inside one window | naive per-SM "
-              "| overlapping windows (coverage, depth min-max) |",
-              "|---|---|---|---|---|---|---|"]
+              "| naive per-warp | overlapping windows (coverage, depth min-max) |",
+              "|---|---|---|---|---|---|---|---|"]
         for name, r in d["windows"].items():
             o = r.get("overlapping")
             ov = (f"{f(o)} ({o['coverage']:.2f}, {o['depth_min']}-{o['depth_max']})" if o else "")
             L.append(f"| {name} | {r['window_gib']:.1f} | {r['coverage']:.2f} | {f(r['grouped'])} | "
                      f"{f(r['unrestricted_inside_one_window'])} | {f(r['naive_per_sm_control'])} "
+                     f"| {f(r['naive_per_warp_control']) if 'naive_per_warp_control' in r else ''} "
                      f"| {ov} |")
         L.append("")
     L += ["## One window per SM, windows spread over the buffer (equal work per SM)", "",

@@ -80,8 +80,10 @@ def test_read_argument_errors_come_before_any_cuda_call():
     assert _call(region_bytes=100) == rr.RR_ERR_RANGE
     assert _call(region_bytes=128 << 32) == rr.RR_ERR_RANGE         # 2^32 lines: one too many
     assert _call(reads_per_warp=1 << 63) == rr.RR_ERR_RANGE
-    # logical mode takes no grouping
+    # logical mode takes no SM grouping; windows alone mean a window per warp
     assert _call(group_of_sm=np.zeros(4, np.uint16), windows=[[0, 8]]) == rr.RR_ERR_ARG
+    assert _call(windows=[[0, 8], [8, 9000]]) == rr.RR_ERR_RANGE
+    assert _call(windows=[[0, 8], [8, 0]]) == rr.RR_ERR_RANGE
     per_sm = dict(mode=rr.RR_MODE_PER_SM, n_warps=0, nsm=4)
     assert _call(warps_per_sm=0, **per_sm) == rr.RR_ERR_ARG
     assert _call(warps_per_sm=65, **per_sm) == rr.RR_ERR_ARG

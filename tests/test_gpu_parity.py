@@ -512,3 +512,19 @@ def test_sorted_variant_grouped_and_pooled(dev, W):
                       warp_start=ws, **kw)
     rr.rr_random_read(p, out, dev.scratch)
     assert np.array_equal(_np(out), oracle.read_pooled(region, W, win, ws, 901, 5))
+
+
+@pytest.mark.parametrize("W", [1, 2, 4])
+@pytest.mark.parametrize("variant", [rr.RR_VARIANT_LDG, rr.RR_VARIANT_PACKED])
+def test_logical_mode_with_a_window_per_warp(dev, W, variant):
+    region = dev.buf_bytes
+    win, cov = rr.rr_make_windows(region, W, region // 7, 37, policy=1, seed=23)   # hashed chunks
+    win[5] = (321, 3)
+    n_warps = 777
+    out = _out(dev, n_warps)
+    p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
+                      reads_per_warp=45, first_read=7, seed=23, windows=win, variant=variant)
+    res = rr.rr_random_read(p, out, dev.scratch)
+    assert res.bytes == n_warps * 45 * 128 * W
+    assert np.array_equal(_np(out), oracle.read_logical_windows(region, W, n_warps, 45, 23, win,
+                                                                first_read=7))

@@ -68,3 +68,19 @@ def test_errors():
         oracle.make_windows(100, 1, 1 << 10, 2)
     with pytest.raises(oracle.OracleError):
         oracle.make_windows(1 << 20, 1, 1 << 10, 0)
+
+
+def test_per_warp_windows_equal_the_per_warp_definition():
+    region = 5000 * 128
+    win, cov = oracle.make_windows(region, 1, 700 * 128, 37, policy=1, seed=23)   # hashed chunks
+    out = oracle.read_logical_windows(region, 1, 100, 9, 23, win, first_read=4)
+    for v in range(100):
+        base, n = map(int, win[v % 37])
+        assert tuple(out[v]) == oracle.warp_checksum(23, v, 4, 9, 1, base, n, n_warps_total=100)
+        for i in range(4, 13):
+            assert base <= oracle.line(23, v, i, base, n) < base + n
+    # one window covering everything: the plain logical mode
+    whole = oracle.read_logical_windows(region, 1, 50, 7, 3, [[0, 5000]])
+    assert np.array_equal(whole, oracle.read_logical(region, 1, 50, 7, 3))
+    with pytest.raises(oracle.OracleError):
+        oracle.read_logical_windows(region, 1, 10, 1, 1, [[4990, 20]])
