@@ -255,7 +255,9 @@ int32_t rr_read_block_times(const void *scratch_dev /*DEVICE*/, uint32_t nsm,
  * For them this entry point performs exactly the read rr_random_read performs, but keeps the
  * claim table, status words and per-block timing records in a fixed array that is part of the
  * library image (RR_STATIC_SCRATCH_BYTES bytes, resident on every GPU that loads the library,
- * until the process exits).  It calls no allocation routine of any kind, and creates no events:
+ * until the process exits).  It allocates no device memory -- no cudaMalloc, cudaFree or other
+ * allocating CUDA or library routine is called (the launch-configuration cache above lives in
+ * host memory) -- and creates no events:
  * res->seconds_event is 0 and res->gbps is computed from the device-side timers.
  *
  * Limit: at most RR_STATIC_MAX_SM SMs (the device's count, or the nsm passed in), and no
