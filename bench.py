@@ -9,8 +9,11 @@ address windows below the measured translation reach, next to the unrestricted r
 One step = one launch of the persistent read kernel over ~95 % of free HBM: 148 x 32 logical
 warps perform 2^8 x 2048 random 128-byte line reads each (about 60 ms of kernel time).  The
 timed workload is the finest static-window policy: every SM reads inside a window of its own,
-the windows of one resource group's SMs lie side by side, all windows together tile the buffer,
-and window size and work follow measured capacity (pooled mode).
+the windows of one resource group's SMs lie side by side, all windows together tile the buffer.
+Two ways of running that policy are measured as arms e and g and the faster one on this card is
+timed (--plan forces one): window size and work in proportion to measured capacity (pooled mode,
+packed kernel), or equal static slices with each warp's reads taken part by part of its slice
+(sorted kernel; the same reads and checksums in another order).
 
 Before the timed region each rank calibrates its own GPU (the layout differs card to card): fill,
 pair-probe matrix, clustering into SM groups, size sweep and reach.  Then every arm of the
@@ -57,6 +60,7 @@ VARIANT_SORTED = 3            # the same, each warp's reads taken part by part o
 UNROLL = 1                    # warp loads in flight per warp (4 lines): with 32 warps per SM and
                               # balanced work a deeper ring only adds power (5654 against 5549 GB/s)
 MOVING_WARPS_PER_SM = 24      # the moving-window arms need fewer warps still (6135 against 5881)
+SORTED = dict(variant=VARIANT_SORTED, unroll=2, sort_parts=16, sort_reads=256)
 SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
@@ -80,17 +84,16 @@ def _sample_warps(n):
     return sorted(set(list(range(0, n, 37)) + [0, n - 1]))
 
 
-def _oracle_all_warps(region_bytes, windows, warp_start, target_seconds):
-    """Times the oracle, as it stands, on all logical warps of the workload for a bounded number
-    of reads per warp.  Returns (GB/s-equivalent, reads_per_warp, seconds, checksums)."""
-    import oracle
-    n_warps = int(warp_start[-1])
+def _oracle_all_warps(run, n_warps, target_seconds):
+    """Times the oracle, as it stands, on all warps of the timed workload for a bounded number
+    of reads per warp; run(reads) calls it.  Returns (GB/s-equivalent, reads_per_warp, seconds,
+    checksums)."""
     t0 = time.time()
-    oracle.read_pooled(region_bytes, 1, windows, warp_start, 8, SEED)
+    run(8)
     per_read = max((time.time() - t0) / 8, 1e-6)
     reads = int(max(8, min(1 << 20, target_seconds / per_read)))
     t0 = time.time()
-    out = oracle.read_pooled(region_bytes, 1, windows, warp_start, reads, SEED)
+    out = run(reads)
     dt = time.time() - t0
     return n_warps * reads * 128 / dt * 1e-9, reads, dt, out
 
@@ -121,7 +124,8 @@ def run_reference(args):
     n_warps = nsm * WARPS_PER_SM
     windows, warp_start = oracle.make_weighted_windows(region, 1, [1000] * nsm, n_warps)
     per_step = max(0.5, min(4.0, 60.0 / max(args.steps + args.warmup, 1)))
-    _, reads, _, _ = _oracle_all_warps(region, windows, warp_start, per_step)
+    _, reads, _, _ = _oracle_all_warps(
+        lambda r: oracle.read_pooled(region, 1, windows, warp_start, r, SEED), n_warps, per_step)
     for k in range(args.warmup):
         oracle.read_pooled(region, 1, windows, warp_start, reads, SEED, first_read=k * reads)
     t0 = time.time()
@@ -347,9 +351,21 @@ def _run_gpu(args, holder):
         pooled(owners.group_of_sm, bal_windows, warp_start, arm_reads), bal_windows, coverage=1.0,
         gbps_by_balancing_round=bal_history)
 
+    # static per-SM slices, equal work, no calibration of weights: the kernel performs each
+    # warp's reads part by part of its window (same reads and checksums, another order)
+    eq_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
+
+    def sorted_static(reads, first_read=0):
+        return ses.params(N, W=1, seed=SEED, reads_per_warp=reads, first_read=first_read,
+                          group_of_sm=owners.group_of_sm, windows=eq_windows, **SORTED)
+
+    arms["g_sorted_execution_static_per_sm_slices"] = measure(
+        sorted_static(arm_reads), eq_windows, coverage=1.0, sort_parts=SORTED["sort_parts"],
+        sort_reads=SORTED["sort_reads"], kernel="read_kernel<U=2, sorted>")
+
     if full:
         # moving windows: the same per-SM slices (equal size, equal work), one sub-window at a time
-        mv_windows, _ = rr.rr_make_weighted_windows(N, 1, [1] * ses.nsm, n_warps, max_window)
+        mv_windows = eq_windows
         slice_bytes = int(mv_windows[:, 1].max()) * 128
         mv_parts, mv_sub = rr.rr_phase_window(slice_bytes, sm_reach, 64)
         phased = dict(index_mode=rr.RR_INDEX_PHASED, phase_reads=1024, phase_window_bytes=mv_sub,
@@ -364,13 +380,6 @@ def _run_gpu(args, holder):
             window_gib_min_max=[N / GiB, N / GiB], coverage=1.0,
             sub_window_mib=mv_sub / (1 << 20), phase_reads=1024, warps_per_sm=MOVING_WARPS_PER_SM,
             note="every SM's window is the whole buffer; SM cycles staggered")
-        # static per-SM slices, equal work, no calibration of weights: the kernel performs each
-        # warp's reads part by part of its window (same reads and checksums, another order)
-        arms["g_sorted_execution_static_per_sm_slices"] = measure(
-            ses.params(N, W=1, seed=SEED, reads_per_warp=arm_reads, group_of_sm=owners.group_of_sm,
-                       windows=mv_windows, variant=VARIANT_SORTED, unroll=1, sort_parts=4,
-                       sort_reads=1024), mv_windows, coverage=1.0, sort_parts=4, sort_reads=1024,
-            kernel="read_kernel<U=1, sorted>")
     t_arms = time.time() - t_arms
     c_head = cfg4[headline]["gbps"]
     comparison = {
@@ -386,13 +395,48 @@ def _run_gpu(args, holder):
     stream = torch.cuda.current_stream()
     step_bytes = n_warps * reads * 128
 
+    # the two ways of running the per-SM-window policy; the faster arm is the one that is timed
+    e_gbps = arms["e_pooled_one_window_per_sm"]["gbps"]
+    g_gbps = arms["g_sorted_execution_static_per_sm_slices"]["gbps"]
+    plan = args.plan
+    if plan == "auto":
+        plan = "sorted" if g_gbps > e_gbps else "pooled"
+    if world > 1:                              # replicas time the same kernel: rank 0's choice
+        pick = torch.tensor([1 if plan == "sorted" else 0], device="cuda")
+        dist.broadcast(pick, 0)
+        plan = "sorted" if pick.item() else "pooled"
+    if plan == "sorted":
+        plan_windows = eq_windows
+        plan_kernel = "read_kernel<W=1, U=2, sorted>: 8 lanes x 16 B per line, per-SM mode"
+
+        def plan_params(n_reads, first_read=0):
+            return sorted_static(n_reads, first_read)
+
+        def window_of_warp(v):                 # warp v runs on SM v // 32
+            return map(int, eq_windows[int(owners.group_of_sm[v // WARPS_PER_SM])])
+
+        def oracle_all_warps(n_reads):
+            return oracle.read_per_sm(N, 1, ses.nsm, WARPS_PER_SM, n_reads, SEED,
+                                      group_of_sm=owners.group_of_sm, windows=eq_windows)
+    else:
+        plan_windows = bal_windows
+        plan_kernel = "read_kernel<W=1, U=1, packed>: 8 lanes x 16 B per line, pooled mode"
+
+        def plan_params(n_reads, first_read=0):
+            return pooled(owners.group_of_sm, bal_windows, warp_start, n_reads, first_read)
+
+        def window_of_warp(v):                 # logical warp v belongs to window g
+            return map(int, bal_windows[int(np.searchsorted(warp_start, v, side="right") - 1)])
+
+        def oracle_all_warps(n_reads):
+            return oracle.read_pooled(N, 1, bal_windows, warp_start, n_reads, SEED)
+
     def step_params(step):
-        return pooled(owners.group_of_sm, bal_windows, warp_start, reads, first_read=step * reads)
+        return plan_params(reads, first_read=step * reads)
 
     def timed_region():
         for _ in range(SETTLE_LAUNCHES):      # untimed: bring clocks to their sustained level
-            rr.rr_random_read(pooled(owners.group_of_sm, bal_windows, warp_start, arm_reads),
-                              ses.out, ses.scratch, timed=False)
+            rr.rr_random_read(plan_params(arm_reads), ses.out, ses.scratch, timed=False)
         for k in range(args.warmup):
             rr.rr_random_read(step_params(k), ses.out, ses.scratch, timed=False)
         torch.cuda.synchronize()
@@ -459,8 +503,7 @@ def _run_gpu(args, holder):
     sample = _sample_warps(n_warps)
     bad = []
     for v in sample:
-        g = int(np.searchsorted(warp_start, v, side="right") - 1)
-        base, n = map(int, bal_windows[g])
+        base, n = window_of_warp(v)
         if tuple(timed_checksums[v]) != oracle.warp_checksum(SEED, v, last_step * reads, reads, 1,
                                                              base, n):
             bad.append(v)
@@ -470,9 +513,8 @@ def _run_gpu(args, holder):
                              "mismatches": len(bad), "oracle_seconds": time.time() - t0}}
     if rank == 0 and world == 1:
         # (2) every logical warp of the same plan on a bounded number of reads (also the CPU timing)
-        o_gbps, o_reads, o_dt, o_out = _oracle_all_warps(N, bal_windows, warp_start, 12.0)
-        rr.rr_random_read(pooled(owners.group_of_sm, bal_windows, warp_start, o_reads), ses.out,
-                          ses.scratch)
+        o_gbps, o_reads, o_dt, o_out = _oracle_all_warps(oracle_all_warps, n_warps, 12.0)
+        rr.rr_random_read(plan_params(o_reads), ses.out, ses.scratch)
         all_same = bool(np.array_equal(ses.checksums(n_warps), o_out))
         parity["all_warps"] = {"warps": n_warps, "reads_per_warp": o_reads, "bit_exact": all_same}
         parity["bit_exact"] = parity["bit_exact"] and all_same
@@ -509,9 +551,14 @@ def _run_gpu(args, holder):
             "config": {
                 "workload": "cfg4 grouped full-memory random 128-B line reads, per-SM-window "
                             "policy: every SM held to its own window inside its resource group's "
-                            "stretch of the buffer, windows tile the buffer, work and window size "
-                            "in proportion to measured capacity (pooled mode), seed 23; the "
-                            "paper's one-window-per-group policy is arms.c / arms.d",
+                            "stretch of the buffer, windows tile the buffer, seed 23; " + (
+                                "equal static slices, each warp's reads performed part by part "
+                                "of its slice (sorted kernel)" if plan == "sorted" else
+                                "work and window size in proportion to measured capacity "
+                                "(pooled mode)") + "; the paper's one-window-per-group policy "
+                            "is arms.c / arms.d",
+                "plan": plan, "plan_requested": args.plan,
+                "plan_candidates_gbps": {"pooled": e_gbps, "sorted": g_gbps},
                 "one_window_per_group_gbps": {"equal_work_per_sm": c_head,
                                               "capacity_weighted": arms.get(
                                                   "d_pooled_one_window_per_group", {}).get("gbps"),
@@ -520,9 +567,9 @@ def _run_gpu(args, holder):
                 "region_bytes": N, "region_gib": N / GiB, "line_bytes": 128,
                 "logical_warps": n_warps, "warps_per_sm": WARPS_PER_SM,
                 "reads_per_warp_per_step": reads,
-                "kernel": "read_kernel<W=1, U=1, packed>: 8 lanes x 16 B per line, pooled mode",
-                "window_gib_min_max": [float(bal_windows[:, 1].min()) * 128 / GiB,
-                                       float(bal_windows[:, 1].max()) * 128 / GiB],
+                "kernel": plan_kernel,
+                "window_gib_min_max": [float(plan_windows[:, 1].min()) * 128 / GiB,
+                                       float(plan_windows[:, 1].max()) * 128 / GiB],
                 "coverage": 1.0, "n_groups": groups.n_groups, "n_windows": owners.n_groups,
                 "l2": "inputs (region) far larger than L2; no flush needed",
                 "parallelism": "replicas" if world > 1 else "single GPU",
@@ -591,6 +638,10 @@ def main():
     ap.add_argument("--clock-period-ms", type=int, default=50,
                     help="period of the nvidia-smi clock sampler; 0 switches it off (do that "
                          "under a profiler)")
+    ap.add_argument("--plan", default="auto", choices=["auto", "pooled", "sorted"],
+                    help="how the timed per-SM-window workload runs: capacity-weighted pooled "
+                         "mode (packed kernel), equal static slices with sorted execution, or "
+                         "whichever of the two measured faster on this card (auto)")
     ap.add_argument("--arms", default="all", choices=["all", "headline"],
                     help="headline: only the arms value and comparison need (a, b, c at the "
                          "headline window, e)")

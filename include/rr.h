@@ -176,7 +176,9 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   warp's window (sort_parts equal parts): at any moment an SM then works inside 1/sort_parts of
  *   its window, which its own translation cache can hold, although the window -- the set of lines
  *   the warp may read, Section 1.3 -- is unchanged and static.  Results are those of
- *   RR_VARIANT_PACKED bit for bit; the price is sort_parts hashes per read.
+ *   RR_VARIANT_PACKED bit for bit; the price is a second hash per read (one pass classifies the
+ *   epoch's reads by part, then each part's reads are hashed again as full vectors) and
+ *   4.75 KB of shared memory per warp.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
@@ -213,9 +215,10 @@ typedef struct {
     uint32_t phase_reads;       /* RR_INDEX_PHASED: reads per phase, a power of two >= 32      */
     uint32_t mix_period;        /* RR_INDEX_MIXED: a power of two in [1, 2^20]; else must be 0  */
     uint64_t phase_window_bytes; /* RR_INDEX_PHASED: largest sub-window                        */
-    uint32_t sort_parts;        /* RR_VARIANT_SORTED: parts of the window, a power of two 2..64 */
+    uint32_t sort_parts;        /* RR_VARIANT_SORTED: parts of the window: 2, 4, 8 or 16         */
     uint32_t sort_reads;        /* RR_VARIANT_SORTED: reads per part and epoch, a multiple of  */
-                                /* 32 (1024 is a good value); both 0 for every other variant   */
+                                /* 32 with sort_parts * sort_reads <= 4096 (16 x 256 is a good */
+                                /* value); both 0 for every other variant                      */
 } rr_read_params_t;
 
 typedef struct {

@@ -3,7 +3,7 @@
     python -m paper_2405_11425_b200.cases read  [--region-gib 4] [--W 1] [--reads 4096]
                                                 [--launches 3] [--groups 0] [--unroll 0]
                                                 [--stride] [--warps-per-sm 32] [--packed] [--pooled]
-                                                [--sorted-parts 4]
+                                                [--sorted-parts 8] [--sorted-reads 512]
     python -m paper_2405_11425_b200.cases fill  [--region-gib 4] [--launches 3]
     python -m paper_2405_11425_b200.cases probe [--region-gib 4] [--reads 65536] [--pairs 4]
     python -m paper_2405_11425_b200.cases cluster [--n 148]
@@ -37,6 +37,8 @@ def main(argv=None):
                     help="logical warps owned by the synthetic groups, work shared inside a group")
     ap.add_argument("--sorted-parts", type=int, default=0,
                     help="sorted execution: one window per SM, reads taken part by part")
+    ap.add_argument("--sorted-reads", type=int, default=0,
+                    help="reads per part and epoch (default 4096 / parts)")
     ap.add_argument("--warps-per-sm", type=int, default=32)
     ap.add_argument("--pairs", type=int, default=4)
     ap.add_argument("--n", type=int, default=148)
@@ -92,12 +94,16 @@ def main(argv=None):
         windows, _ = rr.rr_make_windows(region, a.W, -(-region // a.groups), a.groups)
     o = torch.zeros((nsm * a.warps_per_sm, 2), dtype=torch.int32, device="cuda")
     variant = rr.RR_VARIANT_PACKED if a.packed else rr.RR_VARIANT_LDG
-    if a.sorted_parts:
+    if a.sorted_parts:  # one window per SM, equal work; with --pooled each SM's warps share it
         groups = np.arange(nsm, dtype=np.uint16)
-        windows, _ = rr.rr_make_weighted_windows(region, a.W, [1] * nsm, nsm * a.warps_per_sm)
+        n_warps = nsm * a.warps_per_sm
+        windows, warp_start = rr.rr_make_weighted_windows(region, a.W, [1] * nsm, n_warps)
+        kw = dict(mode=rr.RR_MODE_POOLED, n_warps=n_warps, nsm=nsm,
+                  warp_start=warp_start) if a.pooled else {}
         p = rr.ReadParams(buf, region, W=a.W, warps_per_sm=a.warps_per_sm, reads_per_warp=a.reads,
                           seed=7, unroll=a.unroll, group_of_sm=groups, windows=windows,
-                          variant=rr.RR_VARIANT_SORTED, sort_parts=a.sorted_parts, sort_reads=1024)
+                          variant=rr.RR_VARIANT_SORTED, sort_parts=a.sorted_parts,
+                          sort_reads=a.sorted_reads or 4096 // a.sorted_parts, **kw)
     elif a.pooled:
         import rr_inputs
         n_groups = a.groups or 24

@@ -115,11 +115,31 @@ struct ReadArgs {
 
 constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarSorted = 3;
 
-// Per-warp working memory some variants need beside their registers.
+// Per-warp working memory of the SORTED variant, carved out of the block's dynamic shared memory.
+constexpr uint32_t kSortQueue = 64;       // lines waiting for the load loop: two vectors of 32
+constexpr uint32_t kSortPending = 256;    // reads of the current part waiting to be hashed again
+constexpr uint32_t kSortMaxBatches = 128; // batches of 32 reads per epoch (parts * reads <= 4096)
+constexpr uint32_t kSortMaxBits = 4;      // at most 16 parts
+constexpr uint32_t kSortMaskWords = kSortMaxBits * kSortMaxBatches;  // one epoch's masks
+constexpr uint32_t kSortWarpWords = 2 * kSortMaskWords + kSortPending / 2 + kSortQueue;
+constexpr uint32_t kSortWarpBytes = kSortWarpWords * 4u;
+static_assert(kSortWarpBytes % 16u == 0, "mask words are written in pairs");
 struct WarpScratch {
-    uint32_t *queue;  // SORTED variant: this warp's ring of kSortQueue line indices (shared memory)
+    uint32_t *words;  // this warp's kSortWarpWords words of shared memory (SORTED variant), laid out:
+    // two sets (this epoch's, the next epoch's) of [bit][batch]: bit of the part number of each
+    // of the batch's 32 reads
+    __device__ __forceinline__ uint32_t *mask(uint32_t set) const
+    {
+        return words + set * kSortMaskWords;
+    }
+    // ring of line indices
+    __device__ __forceinline__ uint32_t *queue() const { return words + 2 * kSortMaskWords; }
+    // ring of epoch-relative read numbers
+    __device__ __forceinline__ uint16_t *pending() const
+    {
+        return reinterpret_cast<uint16_t *>(words + 2 * kSortMaskWords + kSortQueue);
+    }
 };
-constexpr uint32_t kSortQueue = 64;  // two vectors of 32 lines
 
 template <int W, int U, bool CHECKED>
 __device__ __forceinline__ void warp_reads_lines(const char *__restrict__ buf, uint64_t region_bytes,
@@ -293,63 +313,188 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
 // Sorted execution of the packed shape.  The checksums do not depend on the order in which a
 // warp performs its reads, so the warp may take them in an order that is kind to the SM's own
 // translation cache: the stream is cut into epochs of P * R reads, and the reads of an epoch are
-// performed part by part of the window (P equal parts), i.e. the warp walks the epoch's indices
-// P times and each time keeps those that fall into the current part.  At any moment the SM is
-// then working inside 1/P of its window.  Same reads, same words, same checksums; the price is
-// P hashes per read instead of one.  Lines that were kept wait in a small ring in shared memory
-// until 32 of them make a vector for the load loop.
+// performed part by part of the window (P parts of equal size).  At any moment the SM is then
+// working inside 1/P of its window.  Same reads, same words, same checksums.
+//
+// Every read is first classified: its part number goes, bit by bit, into ballot masks in shared
+// memory (log2 P words per 32 reads).  Then, part by part, the masks -- one batch per lane, 1024
+// reads at a time -- say which reads belong to the part; their numbers collect in a ring until
+// 32 of them make a full vector, which is hashed again, all lanes busy, into line indices for
+// the load loop.  Two hashes per read whatever P is, plus well under one instruction per read
+// and part for looking at the masks.  The next epoch is classified a little with every vector
+// of the current one (two sets of masks), so that the warps of an SM, which move through the
+// parts together, never all stop loading to classify.
+// Which index belongs to which part is this kernel's own business (any partition gives the same
+// checksums): part = floor(index * P / n) by one multiply.
 struct SortedSource {
-    uint32_t *q;
-    uint32_t head, count;          // ring state, warp-uniform
+    WarpScratch ws;
+    uint32_t head, count;          // line ring, warp-uniform
+    uint32_t phead, pcount;        // pending ring, warp-uniform
     uint64_t epoch0, reads;        // first read of the current epoch (relative), reads of the call
-    uint32_t part, batch;          // current part of the window, batch of 32 candidates inside it
-    uint32_t lo, hi;               // index range of the current part
+    uint32_t in_epoch;             // reads of the current epoch
+    uint32_t next_in;              // reads of the next epoch, 0 when there is none
+    uint32_t next_step;            // pairs of batches of the next epoch classified so far
+    uint32_t part, batch;          // scan position: part of the window, batch of 32 reads
+    uint32_t scale;                // floor(2^32 * P / n), saturated
+    uint32_t cur;                  // which set of masks belongs to the current epoch
     bool done;
-    __device__ __forceinline__ void set_part(uint32_t n, uint32_t shift)
+    __device__ __forceinline__ uint32_t epoch_len(const IndexSpec &ix, uint64_t from) const
     {
-        lo = (uint32_t)(((uint64_t)n * part) >> shift);
-        hi = (uint32_t)(((uint64_t)n * (part + 1)) >> shift);
+        const uint64_t epoch_reads = (uint64_t)ix.sort_reads << ix.sort_shift;
+        const uint64_t left = reads > from ? reads - from : 0;
+        return (uint32_t)(left < epoch_reads ? left : epoch_reads);
     }
-    __device__ __forceinline__ void init(uint32_t *queue, uint64_t reads_, uint32_t n, uint32_t shift)
+    // Part numbers of reads [64 * step, 64 * step + 64) of the epoch that starts at `from`.
+    template <int BITS>
+    __device__ __forceinline__ void classify_step(uint64_t key, uint64_t first, uint64_t from,
+                                                  uint32_t step, uint32_t set, const Divisor &div,
+                                                  uint32_t lane)
     {
-        q = queue;
-        head = count = 0;
+        const uint64_t z = key + (first + from + (step << 6) + lane) * kGamma;
+        uint32_t m[BITS][2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const uint32_t idx = mod_exact(sm64(z + (uint64_t)(32 * j) * kGamma), div);
+            const uint32_t q = min(__umulhi(idx, scale), (1u << BITS) - 1u);
+#pragma unroll
+            for (int k = 0; k < BITS; ++k) m[k][j] = __ballot_sync(0xFFFFFFFFu, (q >> k) & 1u);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int k = 0; k < BITS; ++k)
+                *reinterpret_cast<uint2 *>(ws.mask(set) + k * kSortMaxBatches + (step << 1)) =
+                    make_uint2(m[k][0], m[k][1]);
+        }
+    }
+    __device__ __forceinline__ void classify_step(const IndexSpec &ix, uint64_t key,
+                                                  uint64_t first, uint64_t from, uint32_t step,
+                                                  uint32_t set, const Divisor &div, uint32_t lane)
+    {
+        if (ix.sort_shift == 4) classify_step<4>(key, first, from, step, set, div, lane);
+        else if (ix.sort_shift == 3) classify_step<3>(key, first, from, step, set, div, lane);
+        else if (ix.sort_shift == 2) classify_step<2>(key, first, from, step, set, div, lane);
+        else classify_step<1>(key, first, from, step, set, div, lane);
+    }
+    __device__ __forceinline__ void init(const WarpScratch &ws_, uint64_t reads_, uint32_t n,
+                                         const IndexSpec &ix, uint64_t key, uint64_t first,
+                                         const Divisor &div, uint32_t lane)
+    {
+        ws = ws_;
+        head = count = phead = pcount = 0;
         epoch0 = 0;
         reads = reads_;
         part = batch = 0;
+        cur = 0;
         done = reads_ == 0;
-        set_part(n, shift);
+        const uint64_t sc = (1ull << (32 + ix.sort_shift)) / n;
+        scale = sc > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sc;
+        in_epoch = epoch_len(ix, 0);
+        for (uint32_t step = 0; (step << 6) < in_epoch; ++step)  // the first epoch, all at once
+            classify_step(ix, key, first, 0, step, 0, div, lane);
+        next_in = epoch_len(ix, in_epoch);
+        next_step = 0;
+        __syncwarp();
+    }
+    // The reads of the current part among the next 32 batches go to the pending ring: lane l
+    // looks at batch + l, a prefix sum over the lanes says where its reads go, and it writes
+    // them out bit by bit.  When the ring cannot take them all, the first so many lanes' do.
+    template <int BITS>
+    __device__ __forceinline__ void scan_block(uint32_t lane)
+    {
+        const uint32_t n_batches = (in_epoch + 31u) >> 5;
+        const uint32_t b = batch + lane;
+        uint32_t sel = 0;
+        if (b < n_batches) {
+            const uint32_t rem = in_epoch - (b << 5);
+            sel = rem >= 32u ? 0xFFFFFFFFu : (1u << rem) - 1u;
+#pragma unroll
+            for (int k = 0; k < BITS; ++k) {
+                const uint32_t m = ws.mask(cur)[k * kSortMaxBatches + b];
+                sel &= ((part >> k) & 1u) ? m : ~m;
+            }
+        }
+        uint32_t incl = __popc(sel);
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= (uint32_t)o) incl += up;
+        }
+        // pcount < 32 here, so the ring has room for at least lane 0's batch
+        const uint32_t room = kSortPending - pcount;
+        const uint32_t n_ok = __popc(__ballot_sync(0xFFFFFFFFu, incl <= room));  // a prefix of lanes
+        const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, n_ok - 1u);
+        if (lane < n_ok) {
+            uint32_t at = phead + pcount + incl - __popc(sel);
+            const uint32_t tag = b << 5;
+            while (sel) {
+                const uint32_t bit = __ffs(sel) - 1;
+                sel &= sel - 1u;
+                ws.pending()[at++ & (kSortPending - 1)] = (uint16_t)(tag | bit);
+            }
+        }
+        pcount += total;
+        batch += n_ok;
+        if (batch >= n_batches) {
+            batch = 0;
+            ++part;
+        }
+    }
+    // Hash up to 32 pending reads into lines.
+    __device__ __forceinline__ void flush(uint64_t key, uint64_t first, uint32_t base,
+                                          const Divisor &div, uint32_t lane)
+    {
+        __syncwarp();
+        const uint32_t take = pcount < 32u ? pcount : 32u;
+        if (lane < take) {
+            const uint32_t rel = ws.pending()[(phead + lane) & (kSortPending - 1)];
+            ws.queue()[(head + count + lane) & (kSortQueue - 1)] =
+                base + mod_exact(sm64(key + (first + epoch0 + rel) * kGamma), div);
+        }
+        count += take;
+        phead = (phead + take) & (kSortPending - 1);
+        pcount -= take;
+        __syncwarp();
+    }
+    // One unit of work towards the next vector of lines.
+    __device__ __forceinline__ void work(const IndexSpec &ix, uint64_t key, uint64_t first,
+                                         uint32_t base, const Divisor &div, uint32_t lane)
+    {
+        const uint32_t bits = ix.sort_shift;
+        if (pcount >= 32u || (part == (1u << bits) && pcount)) {
+            flush(key, first, base, div, lane);
+        } else if (part == (1u << bits)) {  // every part scanned and drained: the next epoch
+            if (next_in == 0) {
+                done = true;
+                return;
+            }
+            const uint64_t from = epoch0 + in_epoch;
+            for (; (next_step << 6) < next_in; ++next_step)  // whatever is still unclassified
+                classify_step(ix, key, first, from, next_step, cur ^ 1u, div, lane);
+            __syncwarp();
+            epoch0 = from;
+            in_epoch = next_in;
+            cur ^= 1u;
+            part = batch = 0;
+            next_in = epoch_len(ix, epoch0 + in_epoch);
+            next_step = 0;
+        } else {
+            if (bits == 2) scan_block<2>(lane);
+            else if (bits == 3) scan_block<3>(lane);
+            else if (bits == 4) scan_block<4>(lane);
+            else scan_block<1>(lane);
+        }
     }
     // Next vector of 32 lines (lane j holds the j-th); entries past the end of the call are junk.
     __device__ __forceinline__ uint32_t next(const IndexSpec &ix, uint64_t key, uint64_t first,
-                                             uint32_t base, uint32_t n, const Divisor &div,
-                                             uint32_t lane)
+                                             uint32_t base, const Divisor &div, uint32_t lane)
     {
-        const uint32_t parts = 1u << ix.sort_shift;
-        const uint64_t epoch_reads = (uint64_t)ix.sort_reads << ix.sort_shift;
-        while (count < 32u && !done) {
-            const uint64_t t = epoch0 + ((uint64_t)batch << 5) + lane;   // relative read index
-            const uint32_t idx = mod_exact(sm64(key + (first + t) * kGamma), div);
-            const bool keep = t < reads && idx >= lo && idx < hi;
-            const uint32_t m = __ballot_sync(0xFFFFFFFFu, keep);
-            if (keep) q[(head + count + __popc(m & ((1u << lane) - 1u))) & (kSortQueue - 1)] = base + idx;
-            count += __popc(m);
-            // advance: next batch of this part, else next part, else next epoch
-            ++batch;
-            const uint64_t left = reads - epoch0;                       // reads from this epoch on
-            const uint64_t in_epoch = left < epoch_reads ? left : epoch_reads;
-            if (((uint64_t)batch << 5) >= in_epoch) {
-                batch = 0;
-                if (++part == parts) {
-                    part = 0;
-                    epoch0 += in_epoch;
-                    done = epoch0 >= reads;
-                }
-                set_part(n, ix.sort_shift);
-            }
+        if ((next_step << 6) < next_in) {  // 64 reads of the next epoch for 32 of this one
+            classify_step(ix, key, first, epoch0 + in_epoch, next_step, cur ^ 1u, div, lane);
+            ++next_step;
         }
+        while (count < 32u && !done) work(ix, key, first, base, div, lane);
         __syncwarp();
-        const uint32_t v = q[(head + lane) & (kSortQueue - 1)];
+        const uint32_t v = ws.queue()[(head + lane) & (kSortQueue - 1)];
         const uint32_t take = count < 32u ? count : 32u;
         head = (head + take) & (kSortQueue - 1);
         count -= take;
@@ -370,7 +515,7 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
     static_assert(U >= 1 && U <= NL && (NL % U) == 0, "ring depth must divide a vector");
     const Divisor div = make_divisor(n);
     SortedSource src;
-    src.init(ws.queue, reads, n, ix.sort_shift);
+    src.init(ws, reads, n, ix, key, first, div, lane);
     const uint32_t sub = lane / NL;
     const char *lane_ptr = buf + (lane % NL) * 16u;
     uint32_t d[U][4];
@@ -386,7 +531,7 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
         s += v[2] + v[3];
     };
     const uint64_t n_batches = (reads + 31) >> 5;
-    uint32_t cur = src.next(ix, key, first, base, n, div, lane);
+    uint32_t cur = src.next(ix, key, first, base, div, lane);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         uint32_t line = __shfl_sync(0xFFFFFFFFu, cur, u * P + sub);
@@ -394,7 +539,7 @@ __device__ __forceinline__ void warp_reads_sorted(const char *__restrict__ buf, 
     }
     for (uint64_t b = 0; b < n_batches; ++b) {
         const uint64_t t0 = b << 5;
-        const uint32_t nxt = src.next(ix, key, first, base, n, div, lane);
+        const uint32_t nxt = src.next(ix, key, first, base, div, lane);
         if (t0 + 32 + U * P <= reads) {
 #pragma unroll
             for (int k = 0; k < NL; ++k) {
@@ -447,16 +592,19 @@ __device__ __forceinline__ WarpScratch make_warp_scratch(uint32_t warp)
 {
     WarpScratch ws{nullptr};
     if constexpr (VAR == kVarSorted) {
-        __shared__ uint32_t sh_sort_queue[32 * kSortQueue];
-        ws.queue = sh_sort_queue + warp * kSortQueue;
+        extern __shared__ __align__(16) uint32_t dyn_smem[];  // the host asked for enough
+        ws.words = dyn_smem + warp * kSortWarpWords;
     }
     return ws;
 }
 
-template <int W, int U, int VAR>
+// MODE >= 0 compiles one mode's path only (the SORTED variant, whose long inner loop wants the
+// whole register budget for itself); MODE < 0 takes the mode from the arguments.
+template <int W, int U, int VAR, int MODE = -1>
 __global__ void __launch_bounds__(1024, 1)
     read_kernel(const __grid_constant__ ReadArgs a, const __grid_constant__ Tables tab)
 {
+    const uint32_t mode = MODE >= 0 ? (uint32_t)MODE : a.mode;
     __shared__ uint32_t sh_sm, sh_slot, sh_workers;
     __shared__ uint16_t sh_group[RR_MAX_SM];
     __shared__ rr_window_t sh_win[RR_MAX_GROUPS];
@@ -464,7 +612,7 @@ __global__ void __launch_bounds__(1024, 1)
     ScratchHeader *sc = a.scratch;
     WarpScratch ws = make_warp_scratch<VAR>(warp);
 
-    if (a.mode == RR_MODE_POOLED) {
+    if (mode == RR_MODE_POOLED) {
         // Work sharing inside an SM group: items (logical warp, block of reads) come from the
         // group's counter, so the group's SMs split the group's work however fast each runs.
         if (threadIdx.x == 0) {
@@ -476,70 +624,95 @@ __global__ void __launch_bounds__(1024, 1)
         for (uint32_t k = threadIdx.x; k < a.nsm; k += blockDim.x) sh_group[k] = tab.group_of_sm[k];
         for (uint32_t k = threadIdx.x; k < a.n_groups; k += blockDim.x) sh_win[k] = tab.windows[k];
         __syncthreads();
-        const uint32_t sm = sh_sm, slot = sh_slot;
-        if (slot >= a.cps) return;
-        const uint32_t g = sh_group[sm];
-        if (g == RR_SM_INACTIVE) return;
-        const uint32_t base = sh_win[g].base_line, n = sh_win[g].n_lines;
-        const uint32_t v0 = tab.warp_start[g], cnt = tab.warp_start[g + 1] - v0;
-        // physical warps working for this group: its SMs times the warps of one block
-        if (threadIdx.x == 0) sh_workers = 0;
-        __syncthreads();
+        // What the grab loop needs between two runs of reads lives in shared memory, read
+        // through volatile pointers, so that it holds no registers while the reads run: the
+        // load loop wants them all.
+        __shared__ unsigned long long sh_total, sh_t_start;
+        __shared__ uint32_t sh_pool_workers, sh_v0, sh_g;
+        __shared__ unsigned long long sh_grab[32][2];  // per warp: next read, end of the grab
         {
+            const uint32_t sm = sh_sm, slot = sh_slot;
+            if (slot >= a.cps) return;
+            const uint32_t g = sh_group[sm];
+            if (g == RR_SM_INACTIVE) return;
+            // physical warps working for this group: its SMs times the warps of one block
+            if (threadIdx.x == 0) sh_workers = 0;
+            __syncthreads();
             uint32_t mine = 0;
             for (uint32_t k = threadIdx.x; k < a.nsm; k += blockDim.x) mine += sh_group[k] == g;
             if (mine) atomicAdd(&sh_workers, mine);
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const uint32_t v0 = tab.warp_start[g], cnt = tab.warp_start[g + 1] - v0;
+                sh_g = g;
+                sh_v0 = v0;
+                sh_total = (unsigned long long)cnt * a.reads;
+                sh_pool_workers = sh_workers * a.wpc;
+                sh_t_start = globaltimer();
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        const uint64_t workers = (uint64_t)sh_workers * a.wpc;
+        volatile unsigned long long *grab = sh_grab[warp];
         // The group's work is the line of cnt * reads reads (warp-major).  Grabs shrink as the
         // line runs out (guided self-scheduling): long runs while there is plenty, so the load
         // ring is rarely drained, short ones at the end, so no warp is left with a long tail.
-        const uint64_t total = (uint64_t)cnt * a.reads;
-        uint64_t t_start = 0;
-        if (threadIdx.x == 0) t_start = globaltimer();
+        // A group of one SM needs none of that: its warps get equal shares.
+        // Every new grab of the SORTED variant starts with a burst of classification, hence
+        // its longer grabs.
+        constexpr unsigned long long kGrabCap = VAR == kVarSorted ? (1ull << 20) : 8192ull;
         uint32_t *out_words = reinterpret_cast<uint32_t *>(a.out);
         for (;;) {
+            const uint32_t g = *(volatile uint32_t *)&sh_g;
+            const unsigned long long total = *(volatile unsigned long long *)&sh_total;
             unsigned long long x = 0, len = 0;
             if (lane == 0) {
+                const unsigned long long workers = *(volatile uint32_t *)&sh_pool_workers;
                 const unsigned long long seen =
                     *reinterpret_cast<volatile unsigned long long *>(&sc->pool_next[g]);
                 const unsigned long long left = total > seen ? total - seen : 0;
-                len = left / (2 * workers);
-                len = min(len, 8192ull) & ~31ull;
+                if (workers == a.wpc) {  // the pool is this SM's alone: its warps run alike,
+                    len = ((total + workers - 1) / workers + 31ull) & ~31ull;  // one share each
+                } else {
+                    len = left / (2 * workers);
+                    len = min(len, kGrabCap) & ~31ull;
+                }
                 len = max(len, (unsigned long long)a.pool_block);
                 x = atomicAdd(&sc->pool_next[g], len);
             }
             x = __shfl_sync(0xFFFFFFFFu, x, 0);
             len = __shfl_sync(0xFFFFFFFFu, len, 0);
             if (x >= total) break;
-            const uint64_t end = (x + len < total) ? (uint64_t)(x + len) : total;
-            while (x < end) {  // a grab may run over the end of one logical warp into the next
+            grab[1] = (x + len < total) ? x + len : total;
+            while (x < grab[1]) {  // a grab may run over the end of one logical warp into the next
+                const uint64_t end = grab[1];
                 const uint64_t w = x / a.reads, i0 = x - w * a.reads;
                 const uint64_t n_seg = (end - x < a.reads - i0) ? end - x : a.reads - i0;
-                const uint64_t v = v0 + w;
+                const uint32_t v = *(volatile uint32_t *)&sh_v0 + (uint32_t)w;
+                const uint32_t gg = *(volatile uint32_t *)&sh_g;
+                grab[0] = x + n_seg;
                 uint32_t X, S;
-                warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix,
-                                          v, a.n_warps, a.first_read + i0, n_seg, base, n, lane, X,
-                                          S, &sc->violations, ws);
+                warp_reads<W, U, VAR>(a.buf, a.region_bytes, sm64(a.key_seed ^ v), a.ix, v,
+                                      a.n_warps, a.first_read + i0, n_seg, sh_win[gg].base_line,
+                                      sh_win[gg].n_lines, lane, X, S, &sc->violations, ws);
+                x = grab[0];
                 if (lane == 0) {
-                    atomicXor(&out_words[2 * v], X);
-                    atomicAdd(&out_words[2 * v + 1], S);
+                    const uint32_t vv = *(volatile uint32_t *)&sh_v0 + (uint32_t)((x - 1) / a.reads);
+                    atomicXor(&out_words[2 * vv], X);
+                    atomicAdd(&out_words[2 * vv + 1], S);
                 }
-                x += n_seg;
             }
         }
         __syncthreads();
         if (threadIdx.x == 0) {
             BlockRecord r;
-            r.smid = sm;
-            r.slot = slot;
-            r.t_start = t_start;
+            r.smid = sh_sm;
+            r.slot = sh_slot;
+            r.t_start = sh_t_start;
             r.t_end = globaltimer();
-            sc->rec[sm * a.cps + slot] = r;
+            sc->rec[r.smid * a.cps + r.slot] = r;
             atomicAdd(&sc->blocks_run, 1u);
         }
-    } else if (a.mode == RR_MODE_PER_SM) {
+    } else if (mode == RR_MODE_PER_SM) {
         if (threadIdx.x == 0) {
             uint32_t sm = smid();
             sh_sm = sm;
@@ -706,31 +879,38 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(const __grid_constant__ 
 // ---- host side -------------------------------------------------------------------------------
 typedef void (*ReadKernel)(const ReadArgs, const Tables);
 
-static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant)
+static ReadKernel pick_kernel(uint32_t W, uint32_t U, uint32_t variant, uint32_t mode)
 {
     if (variant == RR_VARIANT_PACKED && W < 4) {  // U counts warp loads of 4/W lines each
-#define RR_PACKED_ROW(W_)                                                               \
-    if (W == W_) switch (U) {                                                           \
-            case 1: return read_kernel<W_, 1, kVarPacked>;                              \
-            case 2: return read_kernel<W_, 2, kVarPacked>;                              \
-            case 4: return read_kernel<W_, 4, kVarPacked>;                              \
-            default: return read_kernel<W_, 8, kVarPacked>;                             \
+#define RR_PACKED_ROW(W_, MODE_)                                                        \
+    if (W == W_ && mode == MODE_) switch (U) {                                          \
+            case 1: return read_kernel<W_, 1, kVarPacked, MODE_>;                       \
+            case 2: return read_kernel<W_, 2, kVarPacked, MODE_>;                       \
+            case 4: return read_kernel<W_, 4, kVarPacked, MODE_>;                       \
+            default: return read_kernel<W_, 8, kVarPacked, MODE_>;                      \
         }
-        RR_PACKED_ROW(1)
-        RR_PACKED_ROW(2)
+        RR_PACKED_ROW(1, RR_MODE_LOGICAL)
+        RR_PACKED_ROW(1, RR_MODE_PER_SM)
+        RR_PACKED_ROW(1, RR_MODE_POOLED)
+        RR_PACKED_ROW(2, RR_MODE_LOGICAL)
+        RR_PACKED_ROW(2, RR_MODE_PER_SM)
+        RR_PACKED_ROW(2, RR_MODE_POOLED)
 #undef RR_PACKED_ROW
     }
     if (variant == RR_VARIANT_SORTED && W < 4) {
-        if (W == 1) switch (U) {
-                case 1: return read_kernel<1, 1, kVarSorted>;
-                case 4: return read_kernel<1, 4, kVarSorted>;
-                default: return read_kernel<1, 2, kVarSorted>;
-            }
-        switch (U) {
-            case 1: return read_kernel<2, 1, kVarSorted>;
-            case 4: return read_kernel<2, 4, kVarSorted>;
-            default: return read_kernel<2, 2, kVarSorted>;
+#define RR_SORTED_ROW(W_, MODE_)                                                        \
+    if (W == W_ && mode == MODE_) switch (U) {                                          \
+            case 1: return read_kernel<W_, 1, kVarSorted, MODE_>;                       \
+            case 4: return read_kernel<W_, 4, kVarSorted, MODE_>;                       \
+            default: return read_kernel<W_, 2, kVarSorted, MODE_>;                      \
         }
+        RR_SORTED_ROW(1, RR_MODE_LOGICAL)
+        RR_SORTED_ROW(1, RR_MODE_PER_SM)
+        RR_SORTED_ROW(1, RR_MODE_POOLED)
+        RR_SORTED_ROW(2, RR_MODE_LOGICAL)
+        RR_SORTED_ROW(2, RR_MODE_PER_SM)
+        RR_SORTED_ROW(2, RR_MODE_POOLED)
+#undef RR_SORTED_ROW
     }
     const bool checked = variant == RR_VARIANT_LDG_CHECKED;
 #define RR_ROW(W_, UMAX_)                                                               \
@@ -769,7 +949,9 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     if (p->variant == RR_VARIANT_SORTED) {
         const uint32_t P = p->sort_parts, R = p->sort_reads;
         if (p->words_per_lane == 4 || p->index_mode != RR_INDEX_RANDOM) return RR_ERR_ARG;
-        if (P < 2 || P > 64 || (P & (P - 1)) || R < 32 || R % 32u || R > (1u << 20)) return RR_ERR_ARG;
+        if (P < 2 || P > (1u << kSortMaxBits) || (P & (P - 1)) || R < 32 || R % 32u ||
+            (uint64_t)P * R > 32ull * kSortMaxBatches)
+            return RR_ERR_ARG;
     } else if (p->sort_parts || p->sort_reads) {
         return RR_ERR_ARG;
     }
@@ -918,6 +1100,16 @@ static int32_t search_ballast(const void *kernel, int block, int want, const Dev
         RR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, kernel, block, smem));
         return RR_OK;
     };
+    {  // registers or threads may already hold residency at `want`: then no ballast at all,
+       // and the SM keeps its shared-memory carve-out small and its L1 large
+        int nb = 0;
+        int32_t rc = blocks_at(0, &nb);
+        if (rc != RR_OK) return rc;
+        if (nb == want) {
+            *smem_out = 0;
+            return RR_OK;
+        }
+    }
     int lo = f.smem_per_sm / (want + 1) - per_block_reserved - stat + 1;
     if (lo < 0) lo = 0;
     const int hi = std::min(most, f.smem_per_sm / want - per_block_reserved - stat);
@@ -931,22 +1123,25 @@ static int32_t search_ballast(const void *kernel, int block, int want, const Dev
         }
         if (nb < want) break;
     }
-    // registers or threads already limit residency below `want`
-    int nb = 0;
-    int32_t rc = blocks_at(0, &nb);
-    if (rc != RR_OK) return rc;
-    if (nb == want) {
-        *smem_out = 0;
-        return RR_OK;
-    }
     set_cuda_error(cudaErrorLaunchOutOfResources, "cannot force the requested blocks per SM");
     return RR_ERR_CUDA;
+}
+
+// The opt-in alone, for launches that do not pin their residency (want == 0).
+static int32_t allow_large_smem(const void *kernel, const DeviceFacts &f)
+{
+    cudaFuncAttributes fa;
+    RR_CUDA(cudaFuncGetAttributes(&fa, kernel));
+    g_n_attribute_sets.fetch_add(1);
+    RR_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 std::max(f.smem_per_block_optin - (int)fa.sharedSizeBytes, 0)));
+    return RR_OK;
 }
 
 template <typename K>
 static int32_t launch_smem(K kernel, int block, int want, const DeviceFacts &f, size_t *smem_out)
 {
-    if (want <= 0) return RR_ERR_ARG;
+    if (want < 0) return RR_ERR_ARG;
     const LaunchKey key{f.device, (const void *)kernel, block, want};
     std::lock_guard<std::mutex> lock(g_launch_mutex);
     for (const LaunchEntry &e : g_launch_cache)
@@ -955,10 +1150,28 @@ static int32_t launch_smem(K kernel, int block, int want, const DeviceFacts &f, 
             return RR_OK;
         }
     size_t smem = 0;
-    int32_t rc = search_ballast((const void *)kernel, block, want, f, &smem);
+    int32_t rc = want ? search_ballast((const void *)kernel, block, want, f, &smem)
+                      : allow_large_smem((const void *)kernel, f);
     if (rc != RR_OK) return rc;
     g_launch_cache.push_back(LaunchEntry{key, smem});
     *smem_out = smem;
+    return RR_OK;
+}
+
+// Dynamic shared memory of one read launch: the ballast that pins the blocks per SM (per-SM and
+// pooled modes), and never less than the variant's own working memory.
+template <typename K>
+static int32_t read_launch_smem(K kernel, const rr_read_params_t *p, uint32_t block,
+                                uint32_t warps_per_block, int want, const DeviceFacts &f,
+                                size_t *smem_out)
+{
+    const size_t need =
+        p->variant == RR_VARIANT_SORTED ? (size_t)warps_per_block * kSortWarpBytes : 0;
+    *smem_out = 0;
+    if (want == 0 && need == 0) return RR_OK;
+    int32_t rc = launch_smem(kernel, (int)block, want, f, smem_out);
+    if (rc != RR_OK) return rc;
+    if (*smem_out < need) *smem_out = need;
     return RR_OK;
 }
 
@@ -1080,15 +1293,14 @@ extern "C" int32_t rr_random_read(const rr_read_params_t *p, void *out_dev, void
     Geometry g;
     rc = geometry(p, f, &g);
     if (rc != RR_OK) return rc;
-    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant);
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant, p->mode);
     if (!kernel) return RR_ERR_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
 
     size_t smem = 0;
-    if (p->mode != RR_MODE_LOGICAL) {
-        rc = launch_smem(kernel, (int)g.block, (int)g.cps, f, &smem);
-        if (rc != RR_OK) return rc;
-    }
+    rc = read_launch_smem(kernel, p, g.block, g.wpc, p->mode == RR_MODE_LOGICAL ? 0 : (int)g.cps, f,
+                          &smem);
+    if (rc != RR_OK) return rc;
 
     ReadArgs a;
     Tables tab;
@@ -1490,17 +1702,15 @@ extern "C" int32_t rr_random_read_static(const rr_read_params_t *p, void *out_de
     rc = geometry(p, f, &g);
     if (rc != RR_OK) return rc;
     if (g.cps != 1 || g.grid > kStaticMaxSm) return RR_ERR_STATIC_LIMIT;
-    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant);
+    ReadKernel kernel = pick_kernel(p->words_per_lane, U, p->variant, p->mode);
     if (!kernel) return RR_ERR_ARG;
     void *scratch = nullptr;
     rc = static_scratch_address(f.device, &scratch);
     if (rc != RR_OK) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     size_t smem = 0;
-    if (p->mode == RR_MODE_PER_SM) {
-        rc = launch_smem(kernel, (int)g.block, 1, f, &smem);
-        if (rc != RR_OK) return rc;
-    }
+    rc = read_launch_smem(kernel, p, g.block, g.wpc, p->mode == RR_MODE_PER_SM ? 1 : 0, f, &smem);
+    if (rc != RR_OK) return rc;
     ReadArgs a;
     Tables tab;
     make_launch_args(p, g, f, out_dev, scratch, &a, &tab);

@@ -233,13 +233,13 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     R["moving_windows_no_partition"] = moving_all
 
     # sorted execution: the same static per-SM slices, equal work, each warp's reads taken part by
-    # part of its window (the indices are hashed once per part)
+    # part of its window (epochs of 4096 reads)
     sorted_rows = []
     for parts in (2, 4, 8):
         for U in (1, 2):
             d = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=owners_eq.group_of_sm,
                        windows=eq_win, variant=rr.RR_VARIANT_SORTED, unroll=U, sort_parts=parts,
-                       sort_reads=1024)
+                       sort_reads=4096 // parts)
             sorted_rows.append({"parts": parts, "unroll": U, **d})
     R["sorted_execution"] = sorted_rows
 

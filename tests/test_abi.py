@@ -62,7 +62,8 @@ def test_read_argument_errors_come_before_any_cuda_call():
     assert _call(mix_period=4) == rr.RR_ERR_ARG                              # only with MIXED
     srt = dict(variant=rr.RR_VARIANT_SORTED, sort_parts=4, sort_reads=64)
     assert _call(**{**srt, "sort_parts": 3}) == rr.RR_ERR_ARG
-    assert _call(**{**srt, "sort_parts": 128}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "sort_parts": 32}) == rr.RR_ERR_ARG
+    assert _call(**{**srt, "sort_parts": 8, "sort_reads": 544}) == rr.RR_ERR_ARG    # 4096 per epoch
     assert _call(**{**srt, "sort_reads": 48}) == rr.RR_ERR_ARG
     assert _call(**{**srt, "sort_reads": 0}) == rr.RR_ERR_ARG
     assert _call(**{**srt, "W": 4}) == rr.RR_ERR_ARG
