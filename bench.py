@@ -67,9 +67,10 @@ NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with n
 NSM_NOMINAL = 148
 # DRAM bytes moved per algorithmic byte by the read kernel: dram__bytes_read.sum +
 # dram__bytes_write.sum over lines x 128 B, from the one-pass ncu capture of the same kernel and
-# plan shape on a 160 GiB region that is summarised in profiles/ (9.93 GB read + 0.004 GB written
-# per 9.932 GB launch; on a 4 GiB region L2 hits bring it down to 0.976).
-TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0
+# plan shape on a 160 GiB region that is summarised in profiles/ (packed pooled: 9.93 GB read +
+# 0.004 GB written per 9.932 GB launch; sorted: 9.88-9.89 GB + 0.004 GB; on a 4 GiB region L2 hits
+# bring it down to 0.976 and 0.80).
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"pooled": 1.0, "sorted": 0.995}
 
 
 def _peaks():
@@ -580,7 +581,7 @@ def _run_gpu(args, holder):
             "gpu_launches": args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind} (copy, read+write)",
-                         "traffic": TRAFFIC_PER_ALGORITHMIC_BYTE * step_bytes,
+                         "traffic": TRAFFIC_PER_ALGORITHMIC_BYTE[plan] * step_bytes,
                          "traffic_kind": "scaled by lines read from the one-pass ncu capture of the "
                                          "same kernel on a 160 GiB region (16384 reads per warp)",
                          "theoretical_gbps": ses.info["theoretical_gbps"],
