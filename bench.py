@@ -60,7 +60,7 @@ VARIANT_SORTED = 3            # the same, each warp's reads taken part by part o
 UNROLL = 1                    # warp loads in flight per warp (4 lines): with 32 warps per SM and
                               # balanced work a deeper ring only adds power (5654 against 5549 GB/s)
 MOVING_WARPS_PER_SM = 24      # the moving-window arms need fewer warps still (6135 against 5881)
-SORTED = dict(variant=VARIANT_SORTED, unroll=2, sort_parts=16, sort_reads=256)
+SORTED = dict(variant=VARIANT_SORTED, unroll=1, sort_parts=16, sort_reads=256)
 SEED = 23                     # configs[4]
 METRIC = "random 128-B line read GB/s over full HBM (grouped vs unrestricted), % of HBM peak"
 NOMINAL_REGION = (int(0.95 * 177.7 * GiB) // 512) * 512   # reference arm with no GPU to ask
@@ -362,7 +362,7 @@ def _run_gpu(args, holder):
 
     arms["g_sorted_execution_static_per_sm_slices"] = measure(
         sorted_static(arm_reads), eq_windows, coverage=1.0, sort_parts=SORTED["sort_parts"],
-        sort_reads=SORTED["sort_reads"], kernel="read_kernel<U=2, sorted>")
+        sort_reads=SORTED["sort_reads"], kernel="read_kernel<U=1, sorted>")
 
     if full:
         # moving windows: the same per-SM slices (equal size, equal work), one sub-window at a time
@@ -408,7 +408,7 @@ def _run_gpu(args, holder):
         plan = "sorted" if pick.item() else "pooled"
     if plan == "sorted":
         plan_windows = eq_windows
-        plan_kernel = "read_kernel<W=1, U=2, sorted>: 8 lanes x 16 B per line, per-SM mode"
+        plan_kernel = "read_kernel<W=1, U=1, sorted>: 8 lanes x 16 B per line, per-SM mode"
 
         def plan_params(n_reads, first_read=0):
             return sorted_static(n_reads, first_read)

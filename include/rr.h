@@ -178,7 +178,7 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   the warp may read, Section 1.3 -- is unchanged and static.  Results are those of
  *   RR_VARIANT_PACKED bit for bit; the price is a second hash per read (one pass classifies the
  *   epoch's reads by part, then each part's reads are hashed again as full vectors) and
- *   4.75 KB of shared memory per warp.
+ *   5.25 KB of shared memory per warp.
  * Reads i in [first_read, first_read + reads_per_warp) of each warp's stream are performed
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered

@@ -117,13 +117,14 @@ constexpr int kVarLdg = 0, kVarChecked = 1, kVarPacked = 2, kVarSorted = 3;
 
 // Per-warp working memory of the SORTED variant, carved out of the block's dynamic shared memory.
 constexpr uint32_t kSortQueue = 64;       // lines waiting for the load loop: two vectors of 32
-constexpr uint32_t kSortPending = 256;    // reads of the current part waiting to be hashed again
+constexpr uint32_t kSortPending = 512;    // reads of the current part waiting to be hashed again
 constexpr uint32_t kSortMaxBatches = 128; // batches of 32 reads per epoch (parts * reads <= 4096)
 constexpr uint32_t kSortMaxBits = 4;      // at most 16 parts
 constexpr uint32_t kSortMaskWords = kSortMaxBits * kSortMaxBatches;  // one epoch's masks
 constexpr uint32_t kSortWarpWords = 2 * kSortMaskWords + kSortPending / 2 + kSortQueue;
 constexpr uint32_t kSortWarpBytes = kSortWarpWords * 4u;
-static_assert(kSortWarpBytes % 16u == 0, "mask words are written in pairs");
+static_assert(kSortWarpBytes % 16u == 0 && kSortMaxBatches % 4u == 0 && kSortPending >= 32u + 128u,
+              "mask words are read four at a time; one lane's four batches always fit the ring");
 struct WarpScratch {
     uint32_t *words;  // this warp's kSortWarpWords words of shared memory (SORTED variant), laid out:
     // two sets (this epoch's, the next epoch's) of [bit][batch]: bit of the part number of each
@@ -317,8 +318,8 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
 // working inside 1/P of its window.  Same reads, same words, same checksums.
 //
 // Every read is first classified: its part number goes, bit by bit, into ballot masks in shared
-// memory (log2 P words per 32 reads).  Then, part by part, the masks -- one batch per lane, 1024
-// reads at a time -- say which reads belong to the part; their numbers collect in a ring until
+// memory (log2 P words per 32 reads).  Then, part by part, the masks -- four batches per lane, a
+// whole epoch at a time -- say which reads belong to the part; their numbers collect in a ring until
 // 32 of them make a full vector, which is hashed again, all lanes busy, into line indices for
 // the load loop.  Two hashes per read whatever P is, plus well under one instruction per read
 // and part for looking at the masks.  The next epoch is classified a little with every vector
@@ -395,45 +396,60 @@ struct SortedSource {
         next_step = 0;
         __syncwarp();
     }
-    // The reads of the current part among the next 32 batches go to the pending ring: lane l
-    // looks at batch + l, a prefix sum over the lanes says where its reads go, and it writes
-    // them out bit by bit.  When the ring cannot take them all, the first so many lanes' do.
+    // The reads of the current part among the next 128 batches (a whole epoch) go to the pending
+    // ring: lane l looks at batches batch + 4l .. + 3, a prefix sum over the lanes says where its
+    // reads go, and it writes them out bit by bit.  When the ring cannot take them all, the
+    // first so many lanes' do, and the next call goes on from there.
     template <int BITS>
     __device__ __forceinline__ void scan_block(uint32_t lane)
     {
         const uint32_t n_batches = (in_epoch + 31u) >> 5;
-        const uint32_t b = batch + lane;
-        uint32_t sel = 0;
-        if (b < n_batches) {
-            const uint32_t rem = in_epoch - (b << 5);
-            sel = rem >= 32u ? 0xFFFFFFFFu : (1u << rem) - 1u;
+        const uint32_t b0 = batch + (lane << 2);  // batch stays a multiple of four
+        uint32_t sel[4] = {0u, 0u, 0u, 0u};
+        if (b0 < n_batches) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t at = (b0 + j) << 5;
+                const uint32_t rem = in_epoch > at ? in_epoch - at : 0u;
+                sel[j] = rem >= 32u ? 0xFFFFFFFFu : (1u << rem) - 1u;
+            }
 #pragma unroll
             for (int k = 0; k < BITS; ++k) {
-                const uint32_t m = ws.mask(cur)[k * kSortMaxBatches + b];
-                sel &= ((part >> k) & 1u) ? m : ~m;
+                const uint4 m = *reinterpret_cast<const uint4 *>(ws.mask(cur) +
+                                                                 k * kSortMaxBatches + b0);
+                const uint32_t flip = ((part >> k) & 1u) ? 0u : 0xFFFFFFFFu;
+                sel[0] &= m.x ^ flip;
+                sel[1] &= m.y ^ flip;
+                sel[2] &= m.z ^ flip;
+                sel[3] &= m.w ^ flip;
             }
         }
-        uint32_t incl = __popc(sel);
+        const uint32_t mine = __popc(sel[0]) + __popc(sel[1]) + __popc(sel[2]) + __popc(sel[3]);
+        uint32_t incl = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
             if (lane >= (uint32_t)o) incl += up;
         }
-        // pcount < 32 here, so the ring has room for at least lane 0's batch
+        // pcount < 32 here, so the ring has room for at least lane 0's four batches
         const uint32_t room = kSortPending - pcount;
         const uint32_t n_ok = __popc(__ballot_sync(0xFFFFFFFFu, incl <= room));  // a prefix of lanes
         const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, n_ok - 1u);
         if (lane < n_ok) {
-            uint32_t at = phead + pcount + incl - __popc(sel);
-            const uint32_t tag = b << 5;
-            while (sel) {
-                const uint32_t bit = __ffs(sel) - 1;
-                sel &= sel - 1u;
-                ws.pending()[at++ & (kSortPending - 1)] = (uint16_t)(tag | bit);
+            uint32_t at = phead + pcount + incl - mine;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t tag = (b0 + j) << 5;
+                uint32_t left = sel[j];
+                while (left) {
+                    const uint32_t bit = __ffs(left) - 1;
+                    left &= left - 1u;
+                    ws.pending()[at++ & (kSortPending - 1)] = (uint16_t)(tag | bit);
+                }
             }
         }
         pcount += total;
-        batch += n_ok;
+        batch += n_ok << 2;
         if (batch >= n_batches) {
             batch = 0;
             ++part;

@@ -220,14 +220,14 @@ def test_pooled_one_window_per_sm_sampled(ses):
 def test_sorted_execution_over_the_whole_buffer_sampled(ses, reads, first):
     # bench.py's arm g and, where it is the faster plan, its timed step: one static slice per SM,
     # equal work, each warp's reads taken in epochs of 16 x 256, part by part of its 1.1 GiB
-    # window, two warp loads in flight; once with a ragged last epoch, once a whole step of 2^19
+    # window, one warp load in flight; once with a ragged last epoch, once a whole step of 2^19
     # reads continuing the stream at a late first_read
     region = ses.region_bytes
     owners = np.arange(ses.nsm, dtype=np.uint16)[::-1].copy()
     win, _ = rr.rr_make_weighted_windows(region, 1, [1] * ses.nsm, ses.nsm * WPS)
     p = ses.params(region, W=1, warps_per_sm=WPS, reads_per_warp=reads, first_read=first,
                    seed=rr_inputs.CFG4_SEED, group_of_sm=owners, windows=win,
-                   variant=rr.RR_VARIANT_SORTED, unroll=2, sort_parts=16, sort_reads=256)
+                   variant=rr.RR_VARIANT_SORTED, unroll=1, sort_parts=16, sort_reads=256)
     assert rr.rr_random_read(p, ses.out, ses.scratch, timed=False) is None   # as bench launches it
     res = rr.rr_read_report(p, ses.scratch)
     assert res.sms_covered == ses.nsm and res.bytes == ses.nsm * WPS * reads * 128
