@@ -68,9 +68,9 @@ NSM_NOMINAL = 148
 # DRAM bytes moved per algorithmic byte by the read kernel: dram__bytes_read.sum +
 # dram__bytes_write.sum over lines x 128 B, from the one-pass ncu capture of the same kernel and
 # plan shape on a 160 GiB region that is summarised in profiles/ (packed pooled: 9.93 GB read +
-# 0.004 GB written per 9.932 GB launch; sorted: 9.88-9.89 GB + 0.004 GB; on a 4 GiB region L2 hits
+# 0.004 GB written per 9.932 GB launch; sorted: 9.89 GB + 0.003 GB; on a 4 GiB region L2 hits
 # bring it down to 0.976 and 0.80).
-TRAFFIC_PER_ALGORITHMIC_BYTE = {"pooled": 1.0, "sorted": 0.995}
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"pooled": 1.0, "sorted": 0.996}
 
 
 def _peaks():
