@@ -156,7 +156,7 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  *   read inside windows[g].  The group's work is the line of its warps' reads; the persistent
  *   blocks of the group's SMs (warps_per_sm physical warps each) grab runs of that line from a
  *   per-group counter -- long runs at first, never shorter than pool_block_reads at the end --
- *   until it is used up.  A group with more SMs then does not do more work than its shared
+ *   until it is used up (a group of one SM is simply split into equal shares, one per warp).  A group with more SMs then does not do more work than its shared
  *   translation path can carry, and no group becomes the straggler when warp_start follows the
  *   groups' capacities (rr_make_weighted_windows).  out has n_warps entries, accumulated with
  *   atomics (the call clears it first); the checksums do not depend on which SM did what.

@@ -233,12 +233,14 @@ def run(out_dir: Path, quick: bool = False, alloc_study: bool = False) -> dict:
     R["moving_windows_no_partition"] = moving_all
 
     # sorted execution: the same static per-SM slices, equal work, each warp's reads taken part by
-    # part of its window (epochs of 4096 reads)
+    # part of its window (epochs of 4096 reads), in launches of the benchmark's step size: the
+    # warps of an SM start every launch on the same part and stay together through it
     sorted_rows = []
-    for parts in (2, 4, 8):
+    for parts in (4, 8, 16):
         for U in (1, 2):
-            d = _stats(ses, N, 3, seed=23, reads_per_warp=reads, group_of_sm=owners_eq.group_of_sm,
-                       windows=eq_win, variant=rr.RR_VARIANT_SORTED, unroll=U, sort_parts=parts,
+            d = _stats(ses, N, 3, settle=20, min_ms=500.0, seed=23, reads_per_warp=1 << 19,
+                       group_of_sm=owners_eq.group_of_sm, windows=eq_win,
+                       variant=rr.RR_VARIANT_SORTED, unroll=U, sort_parts=parts,
                        sort_reads=4096 // parts)
             sorted_rows.append({"parts": parts, "unroll": U, **d})
     R["sorted_execution"] = sorted_rows
@@ -369,10 +371,12 @@ def markdown(R: dict) -> str:
         L.append(f"| {r['sub_window_mib']} | {r['phase_reads']} | {r['sustained_gbps']:.0f} |")
     L.append("")
     if "sorted_execution" in R:
-        L += ["## Sorted execution: static per-SM slices, equal work, reads taken part by part", "",
-              "| parts | warp loads in flight | GB/s |", "|---|---|---|"]
+        L += ["## Sorted execution: static per-SM slices, equal work, reads taken part by part "
+              "(2^19 reads per warp and launch)", "",
+              "| parts | reads per part and epoch | warp loads in flight | GB/s |",
+              "|---|---|---|---|"]
         for r in R["sorted_execution"]:
-            L.append(f"| {r['parts']} | {r['unroll']} | {f(r)} |")
+            L.append(f"| {r['parts']} | {4096 // r['parts']} | {r['unroll']} | {f(r)} |")
         L.append("")
     L += ["## Work in proportion to group capacity (pooled mode, windows tile the buffer)", "",
           "| workload | first launch after 1 s idle, GB/s | sustained GB/s (500 launches) | windows GiB |", "|---|---|---|---|"]
