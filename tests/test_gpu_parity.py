@@ -333,6 +333,31 @@ def test_pooled_mode_empty_group_and_zero_reads(dev):
     assert not _np(out).any()
 
 
+@pytest.mark.parametrize("wps", [32, 24, 5])
+@pytest.mark.parametrize("variant", ["ldg", "packed", "sorted"])
+def test_pooled_mode_one_sm_per_group_equal_shares(dev, variant, wps):
+    """A pool that a single SM serves is cut into equal shares, one per warp (no guided grabs):
+    shares that are not whole logical warps, a last share that is short, pools with fewer
+    reads than warps."""
+    region = 600 * MiB + 256
+    owners = np.random.default_rng(5).permutation(dev.nsm).astype(np.uint16)
+    weights = [3 + (g * 7) % 3 for g in range(dev.nsm)]
+    kw = {"ldg": dict(variant=rr.RR_VARIANT_LDG),
+          "packed": dict(variant=rr.RR_VARIANT_PACKED, unroll=1),
+          "sorted": dict(variant=rr.RR_VARIANT_SORTED, unroll=1, sort_parts=16, sort_reads=64)}[variant]
+    for n_warps, reads, first in [(dev.nsm * 3 + 1, 333, 5), (dev.nsm * 2, 1, 0),
+                                  (dev.nsm * 4 + 9, 4099, 64)]:
+        win, ws = rr.rr_make_weighted_windows(region, 1, weights, n_warps)
+        out = _out(dev, n_warps)
+        p = rr.ReadParams(dev.buf, region, W=1, mode=rr.RR_MODE_POOLED, n_warps=n_warps,
+                          warps_per_sm=wps, nsm=dev.nsm, reads_per_warp=reads, first_read=first,
+                          seed=23, group_of_sm=owners, windows=win, warp_start=ws, **kw)
+        res = rr.rr_random_read(p, out, dev.scratch)
+        expect = oracle.read_pooled(region, 1, win, ws, reads, 23, first_read=first)
+        assert np.array_equal(_np(out), expect), (variant, wps, n_warps, reads)
+        assert res.bytes == n_warps * reads * 128 and res.sms_covered == dev.nsm
+
+
 @pytest.mark.parametrize("W", [1, 2, 4])
 @pytest.mark.parametrize("unroll", [0, 2, 4, 8, 16])
 def test_packed_variant_logical_ragged_reads(dev, W, unroll):
