@@ -488,7 +488,10 @@ def _run_gpu(args, holder):
         torch.cuda.synchronize()
     e2e_seconds = time.perf_counter() - t0
     e2e_bytes, e2e_max = aggregate_throughput(step_bytes * e2e_steps, e2e_seconds)
-    h2d = ses.nsm * 2 + owners.n_groups * 12 + 4 + 128     # tables + scalars in the launch
+    # tables + scalars in the launch: SM -> window map, windows, (pooled) warp ranges
+    h2d = ses.nsm * 2 + owners.n_groups * 8 + 128
+    if plan == "pooled":
+        h2d += (owners.n_groups + 1) * 4
     d2h = host_out.numel() * 4 + 8208                      # checksums + timing records
 
     # ---- oracle beside it: parity of the timed workload, and its timing ---------------------------------
