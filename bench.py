@@ -7,7 +7,7 @@ Metric: random 128-B line read GB/s over the full HBM with SM groups held to
 address windows below the measured translation reach, next to the unrestricted rate.
 
 One step = one launch of the persistent read kernel over ~95 % of free HBM: 148 x 32 logical
-warps perform 2^8 x 2048 random 128-byte line reads each (about 60 ms of kernel time).  The
+warps perform 2^8 x 2048 random 128-byte line reads each (53-56 ms of kernel time).  The
 timed workload is the finest static-window policy: every SM reads inside a window of its own,
 the windows of one resource group's SMs lie side by side, all windows together tile the buffer.
 Two ways of running that policy are measured as arms e and g and the faster one on this card is
