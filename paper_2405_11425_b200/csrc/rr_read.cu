@@ -319,9 +319,9 @@ __device__ __forceinline__ void warp_reads_packed(const char *__restrict__ buf, 
 //
 // Every read is first classified: its part number goes, bit by bit, into ballot masks in shared
 // memory (log2 P words per 32 reads).  Then, part by part, the masks -- four batches per lane, a
-// whole epoch at a time -- say which reads belong to the part; their numbers collect in a ring until
-// 32 of them make a full vector, which is hashed again, all lanes busy, into line indices for
-// the load loop.  Two hashes per read whatever P is, plus well under one instruction per read
+// whole epoch at a time -- say which reads belong to the part; their numbers collect in a ring
+// until 32 of them make a full vector, which is hashed again, all lanes busy, into line indices
+// for the load loop.  Two hashes per read whatever P is, plus well under one instruction per read
 // and part for looking at the masks.  The next epoch is classified a little with every vector
 // of the current one (two sets of masks), so that the warps of an SM, which move through the
 // parts together, never all stop loading to classify.
