@@ -183,7 +183,8 @@ int32_t rr_fill(void *buf /*DEVICE*/, uint64_t n_words, void *stream);
  * (reads_per_warp = 0 is valid: all checksums {0,0}).
  * unroll: independent loads kept in flight per warp: 0 (= default 8) or 2, 4, 8, 16, lowered
  *   so that unroll * W <= 32 (the ring lives in registers).  RR_VARIANT_PACKED counts warp
- *   loads of 4/W lines each (1, 2, 4 or 8; default 4).
+ *   loads of 4/W lines each (1, 2, 4 or 8; default 4), RR_VARIANT_SORTED likewise (1, 2 or 4;
+ *   default 1, which measured fastest: the order already shortens the latency to be covered).
  *
  * out_dev (DEVICE, 8-byte aligned): pairs {X, S} of uint32.  scratch_dev: rr_scratch_bytes().
  * res == NULL: asynchronous on `stream`, no timing; decode the scratch later with

@@ -986,7 +986,8 @@ static int32_t validate_read(const rr_read_params_t *p, const void *out, const v
     }
     if (p->mode != RR_MODE_POOLED && (p->pool_block_reads || p->warp_start)) return RR_ERR_ARG;
     const bool packed_shape = p->variant == RR_VARIANT_PACKED || p->variant == RR_VARIANT_SORTED;
-    uint32_t U = p->unroll ? p->unroll : (p->variant == RR_VARIANT_SORTED ? 2u : packed_shape ? 4u : 8u);
+    uint32_t U = p->unroll;
+    if (U == 0) U = p->variant == RR_VARIANT_SORTED ? 1u : packed_shape ? 4u : 8u;
     if (U != 2 && U != 4 && U != 8 && U != 16 && !(U == 1 && packed_shape)) return RR_ERR_ARG;
     if (p->variant == RR_VARIANT_SORTED && U > 4) return RR_ERR_ARG;
     if (U * p->words_per_lane > 32) U = 32 / p->words_per_lane;  // the ring holds 32 words a lane
