@@ -540,15 +540,19 @@ def test_sorted_variant_grouped_and_pooled(dev, W):
 
 
 @pytest.mark.parametrize("W", [1, 2, 4])
-@pytest.mark.parametrize("variant", [rr.RR_VARIANT_LDG, rr.RR_VARIANT_PACKED])
+@pytest.mark.parametrize("variant", [rr.RR_VARIANT_LDG, rr.RR_VARIANT_PACKED,
+                                     rr.RR_VARIANT_SORTED])
 def test_logical_mode_with_a_window_per_warp(dev, W, variant):
+    if variant == rr.RR_VARIANT_SORTED and W == 4:
+        pytest.skip("16-byte lanes already cover a 512-byte line: no packed or sorted shape")
+    kw = dict(sort_parts=8, sort_reads=32) if variant == rr.RR_VARIANT_SORTED else {}
     region = dev.buf_bytes
     win, cov = rr.rr_make_windows(region, W, region // 7, 37, policy=1, seed=23)   # hashed chunks
     win[5] = (321, 3)
     n_warps = 777
     out = _out(dev, n_warps)
     p = rr.ReadParams(dev.buf, region, W=W, mode=rr.RR_MODE_LOGICAL, n_warps=n_warps,
-                      reads_per_warp=45, first_read=7, seed=23, windows=win, variant=variant)
+                      reads_per_warp=45, first_read=7, seed=23, windows=win, variant=variant, **kw)
     res = rr.rr_random_read(p, out, dev.scratch)
     assert res.bytes == n_warps * 45 * 128 * W
     assert np.array_equal(_np(out), oracle.read_logical_windows(region, W, n_warps, 45, 23, win,
